@@ -1,0 +1,164 @@
+/*
+ * pulseinfer.h - C ABI of the B200 (sm_100a) decode recall path of sparse KV-cache
+ * offloading:  score -> top-k select -> miss diff -> gather-scatter recall ->
+ * sparse GQA decode attention, one call per step, per layer, for a whole batch.
+ *
+ * Conventions (all entry points)
+ *   - "dev" pointers are device memory, "pinned" pointers are page-locked host
+ *     memory that the GPU can address (cudaHostAlloc / cudaHostRegister), "host"
+ *     pointers are ordinary host memory.  The caller owns every buffer; the library
+ *     allocates only the small scratch held by pi_ctx.  Buffers must stay alive
+ *     until the stream has drained.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue work and return;
+ *     none of the four path calls synchronises the host.
+ *   - All per-layer arrays are passed by their per-layer base; `layer` only selects
+ *     the retrieval head solo_head[layer].
+ *   - Return value: PI_OK or a negative PI_ERR_* code; nothing is launched when an
+ *     argument check fails.  Problems only the device can see (an index out of
+ *     range, a list longer than its capacity, a bounded wait that ran out, a pool
+ *     with too few evictable slots) set a sticky status word read by pi_get_status;
+ *     the offending access is skipped, never trapped.
+ *   - Shapes use: Hq query heads, Hkv KV heads, G = Hq/Hkv, D = head_dim = 128,
+ *     B = block_tokens, K = budget_blocks, C = pool_slots, NB = max_blocks.
+ *     frag_bytes = B*D*2*2 (K and V of one KV head of one block; 8 KB at B = 16),
+ *     block_bytes = Hkv*frag_bytes.  bf16 everywhere for q, K, V, digests, out.
+ *   - Layout of one block, in the host store and in the pool alike:
+ *     [Hkv][2 = K,V][B][D] bf16, so one (block, head) fragment is contiguous.
+ */
+#ifndef PULSEINFER_H
+#define PULSEINFER_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PI_OK                   0
+#define PI_ERR_INVALID_ARG     (-1)
+#define PI_ERR_BAD_ALIGN       (-2)   /* a pointer is not 16-byte aligned            */
+#define PI_ERR_UNSUPPORTED_DIM (-3)
+#define PI_ERR_POOL_TOO_SMALL  (-4)   /* fewer evictable slots than misses           */
+#define PI_ERR_NOT_PINNED      (-5)   /* host KV store is not GPU-addressable        */
+#define PI_ERR_CUDA            (-6)   /* a CUDA runtime call failed                  */
+#define PI_ERR_TIMEOUT         (-7)   /* a bounded device-side wait ran out          */
+#define PI_ERR_INDEX_RANGE     (-8)   /* a block / slot index read from a list is out of range */
+#define PI_ERR_CAPACITY        (-9)   /* a count read from device memory exceeds its capacity  */
+
+typedef struct pi_ctx pi_ctx;
+
+typedef struct {
+    int32_t n_layers;
+    int32_t n_q_heads, n_kv_heads, head_dim;  /* head_dim must be 128; Hq % Hkv == 0; G <= 16; Hkv <= 16 */
+    int32_t block_tokens;                     /* 16, 32 or 64                                      */
+    int32_t budget_blocks;                    /* K: sink + local + middle blocks per (seq, layer) */
+    int32_t n_sink_blocks, n_local_blocks;    /* always-resident, always-selected prefix / suffix */
+    int32_t pool_slots;                       /* C per (seq, layer); C >= K                       */
+    int32_t max_batch, max_blocks;            /* capacities: batch <= max_batch, NB = max_blocks  */
+    int32_t recall_ctas;                      /* CTAs of the recall kernel, 0 = default           */
+    int32_t attn_ctas;                        /* CTAs of the attention kernel, 0 = one per SM     */
+    const int32_t* solo_head;                 /* host [n_layers]: retrieval KV head per layer (copied) */
+} pi_config;
+
+/* One transfer of the recall list: n_units consecutive units of the host store
+ * starting at src_unit go to n_units consecutive units of the pool starting at
+ * dst_unit.  A unit is `unit_bytes` long (a whole block for the shared selection,
+ * one (block, head) fragment for per-head lists); indices are relative to the
+ * sequence's base.  units_before = units of the earlier extents of the same list. */
+typedef struct {
+    int32_t src_unit, dst_unit, n_units, units_before;
+} pi_extent;
+
+/* Create / destroy the context (device scratch for scores, split-K partials and
+ * completion counters; a pinned status word).  Uses the current CUDA device. */
+int pi_create(const pi_config* cfg, pi_ctx** out);
+int pi_destroy(pi_ctx* ctx);
+
+/* Step 1+2 of the offloading workflow (Sec. 2.2, sparse selection) with the shared
+ * single-head selection of Sec. 4.4.1: score every block of every sequence against
+ * the digest of the layer's retrieval head, keep the sink and local blocks, add the
+ * K - n_sink - n_local best middle blocks (ties to the lower block index).
+ *   q_dev       [batch][Hq][D] bf16           (only the G heads of solo_head[layer] are read)
+ *   digest_dev  [batch][NB][2][D] bf16        row 0 = channel-wise min, row 1 = max of the block's keys
+ *   ctx_len_dev [batch] int32                 tokens per sequence; n_blocks = ceil(ctx/B) <= NB
+ *   sel_blocks_dev [batch][K] int32 (out)     ascending block indices, -1 padded
+ *   sel_count_dev  [batch] int32 (out)
+ *   scores_dev  [batch][NB] float (out) or NULL: score = sum_d Q+[d]*max[d] + Q-[d]*min[d]
+ *               with Q+/- the sums of the positive / negative parts of the group's queries. */
+int pi_score_select(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* digest_dev,
+                    const int32_t* ctx_len_dev, int32_t* sel_blocks_dev, int32_t* sel_count_dev,
+                    float* scores_dev, void* stream);
+
+/* Step 2 of the workflow (Sec. 2.2): B_recall = B_topk \ B_gpu against the
+ * device-resident block table, victim choice (least recently selected slot, ties to
+ * the lower slot; sink / local / selected blocks are never evicted), table update,
+ * and the recall list with adjacent (block, slot) pairs merged into extents.
+ *   step             decode step counter, >= 1, written as the stamp of every selected slot
+ *   block_table_dev  [batch][NB] int32 (in/out)  slot of each block or -1
+ *   slot_block_dev   [batch][C] int32 (in/out)   block held by each slot or -1
+ *   slot_stamp_dev   [batch][C] uint32 (in/out)  step the slot was last selected (0 = never)
+ *   sel_slots_dev    [batch][K] int32 (out)      pool slot of every selected block, -1 padded
+ *   recall_list_dev  [batch][K] pi_extent (out)  units are whole blocks, ascending src_unit
+ *   recall_count_dev [batch] int32 (out)         extents per sequence
+ * A sequence with too few evictable slots keeps its tables, gets recall count 0 and
+ * -1 for its missing blocks in sel_slots, and sets PI_ERR_POOL_TOO_SMALL in the status. */
+int pi_diff_misses(pi_ctx* ctx, int layer, int batch, uint32_t step, const int32_t* ctx_len_dev,
+                   const int32_t* sel_blocks_dev, const int32_t* sel_count_dev,
+                   int32_t* block_table_dev, int32_t* slot_block_dev, uint32_t* slot_stamp_dev,
+                   int32_t* sel_slots_dev, pi_extent* recall_list_dev, int32_t* recall_count_dev,
+                   void* stream);
+
+/* Step 3 of the workflow (Sec. 2.2; Sec. 4.4.2 gather-scatter transfer): copy every
+ * extent of every list from the pinned host store into the HBM pool, byte for byte.
+ * The GPU pulls the data itself with wide loads; counts and lists are read from
+ * device memory, so no host round trip separates this call from pi_diff_misses.
+ *   n_lists, lists_per_seq   list i belongs to sequence i / lists_per_seq (1 for the shared
+ *                            selection, Hkv for per-head lists)
+ *   host_kv_pinned           sequence s starts at host_kv_pinned + s*host_seq_stride_bytes
+ *   pool_dev                 sequence s starts at pool_dev + s*pool_seq_stride_bytes
+ *   recall_list_dev          [n_lists][list_capacity] pi_extent; recall_count_dev [n_lists]
+ *   unit_bytes               multiple of 4096 */
+int pi_recall_gather_scatter(pi_ctx* ctx, int layer, int n_lists, int lists_per_seq,
+                             const void* host_kv_pinned, int64_t host_seq_stride_bytes,
+                             void* pool_dev, int64_t pool_seq_stride_bytes,
+                             const pi_extent* recall_list_dev, int32_t list_capacity,
+                             const int32_t* recall_count_dev, int64_t unit_bytes, void* stream);
+
+/* Attention of the layer over the selected blocks only (Sec. 4.2.1: after the recall
+ * completes the offload batch attends over the recalled blocks): for every query
+ * head, softmax(q.K^T / sqrt(D)) V over the tokens t < ctx_len of the selected blocks,
+ * K/V read from the pool through sel_slots.
+ *   pool_dev [batch][C] blocks; sel_slots_dev / sel_blocks_dev [batch][K]; sel_count_dev [batch]
+ *   out_dev  [batch][Hq][D] bf16 (out);  lse_dev [batch][Hq] float natural-log-sum-exp (out) or NULL
+ * Pool bytes of tokens beyond ctx_len in a selected block must be finite numbers. */
+int pi_sparse_decode_attn(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* pool_dev,
+                          const int32_t* sel_slots_dev, const int32_t* sel_blocks_dev,
+                          const int32_t* sel_count_dev, const int32_t* ctx_len_dev, void* out_dev,
+                          float* lse_dev, void* stream);
+
+/* Helpers around the path (input preparation and measurement; not hot calls).
+ * pi_build_digests: channel-wise min / max of the keys of head solo_head[layer] over the
+ *   valid tokens of each block; kv may be device memory or pinned host memory laid out
+ *   [batch][NB] blocks with the given sequence stride.  Exact: no rounding happens.
+ * pi_table_init: slot i of sequence s holds block resident_dev[s][i] (-1 = free);
+ *   fills block_table, slot_block and zero stamps.
+ * pi_h2d_copy_ms: best time in ms of `reps` cudaMemcpyAsync copies of `bytes` from pinned
+ *   host to device memory (the link's reference bandwidth). Synchronises. */
+int pi_build_digests(pi_ctx* ctx, int layer, int batch, const void* kv, int64_t kv_seq_stride_bytes,
+                     const int32_t* ctx_len_dev, void* digest_dev, void* stream);
+int pi_table_init(pi_ctx* ctx, int batch, const int32_t* resident_dev, int32_t* block_table_dev,
+                  int32_t* slot_block_dev, uint32_t* slot_stamp_dev, void* stream);
+int pi_h2d_copy_ms(const void* host_pinned, void* dev, int64_t bytes, int reps, float* best_ms);
+
+/* Sticky device status.  out[0] = first PI_ERR_* code seen by a kernel (0 = none),
+ * out[1] = stage (1 score/select, 2 diff, 3 recall, 4 attention), out[2..4] = sequence
+ * or list, position, offending value.  Reads a pinned mirror: call after the stream
+ * has been synchronised.  pi_clear_status resets it. */
+int pi_get_status(pi_ctx* ctx, int32_t out[8]);
+int pi_clear_status(pi_ctx* ctx);
+const char* pi_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PULSEINFER_H */

@@ -1,0 +1,211 @@
+"""Thin ctypes binding of the C ABI in include/pulseinfer.h.
+
+Argument marshalling only: tensors are checked (dtype, device, contiguity) and handed
+over as raw pointers; every step of the path runs in the CUDA library.  There is no
+fallback: a missing library or a failing call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from ctypes import POINTER, c_char_p, c_float, c_int, c_int32, c_int64, c_uint32, c_void_p
+from typing import Optional, Sequence
+
+import torch
+
+from .build import LIB, build
+
+OK = 0
+ERR_NAMES = {
+    -1: "PI_ERR_INVALID_ARG", -2: "PI_ERR_BAD_ALIGN", -3: "PI_ERR_UNSUPPORTED_DIM",
+    -4: "PI_ERR_POOL_TOO_SMALL", -5: "PI_ERR_NOT_PINNED", -6: "PI_ERR_CUDA", -7: "PI_ERR_TIMEOUT",
+    -8: "PI_ERR_INDEX_RANGE", -9: "PI_ERR_CAPACITY",
+}
+EXTENT_DTYPE = torch.int32      # a pi_extent is four int32: src_unit, dst_unit, n_units, units_before
+
+EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_diff_misses", "pi_recall_gather_scatter",
+           "pi_sparse_decode_attn", "pi_build_digests", "pi_table_init", "pi_h2d_copy_ms",
+           "pi_get_status", "pi_clear_status", "pi_strerror"]
+
+
+class PiConfig(ctypes.Structure):
+    _fields_ = [("n_layers", c_int32), ("n_q_heads", c_int32), ("n_kv_heads", c_int32), ("head_dim", c_int32),
+                ("block_tokens", c_int32), ("budget_blocks", c_int32), ("n_sink_blocks", c_int32),
+                ("n_local_blocks", c_int32), ("pool_slots", c_int32), ("max_batch", c_int32),
+                ("max_blocks", c_int32), ("recall_ctas", c_int32), ("attn_ctas", c_int32),
+                ("solo_head", POINTER(c_int32))]
+
+
+class PiError(RuntimeError):
+    def __init__(self, call: str, code: int, text: str):
+        super().__init__(f"{call} failed: {ERR_NAMES.get(code, code)} ({text})")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library(rebuild: bool = False) -> ctypes.CDLL:
+    """Loads (building first if the sources are newer) the CUDA library.  Raises if it
+    cannot be built or loaded: there is no other implementation to fall back to."""
+    global _lib
+    if _lib is not None and not rebuild:
+        return _lib
+    path = build(force=rebuild)
+    lib = ctypes.CDLL(str(path))
+    vp, i32p, u32p = c_void_p, c_void_p, c_void_p
+    lib.pi_create.argtypes = [POINTER(PiConfig), POINTER(c_void_p)]
+    lib.pi_destroy.argtypes = [c_void_p]
+    lib.pi_score_select.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, vp, vp]
+    lib.pi_diff_misses.argtypes = [c_void_p, c_int, c_int, c_uint32, i32p, i32p, i32p, i32p, i32p, u32p, i32p, vp, i32p, vp]
+    lib.pi_recall_gather_scatter.argtypes = [c_void_p, c_int, c_int, c_int, vp, c_int64, vp, c_int64, vp, c_int32, i32p, c_int64, vp]
+    lib.pi_sparse_decode_attn.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, i32p, vp, vp, vp]
+    lib.pi_build_digests.argtypes = [c_void_p, c_int, c_int, vp, c_int64, i32p, vp, vp]
+    lib.pi_table_init.argtypes = [c_void_p, c_int, i32p, i32p, i32p, u32p, vp]
+    lib.pi_h2d_copy_ms.argtypes = [vp, vp, c_int64, c_int, POINTER(c_float)]
+    lib.pi_get_status.argtypes = [c_void_p, POINTER(c_int32 * 8)]
+    lib.pi_clear_status.argtypes = [c_void_p]
+    lib.pi_strerror.argtypes = [c_int]
+    lib.pi_strerror.restype = c_char_p
+    for name in EXPORTS:
+        if name != "pi_strerror":
+            getattr(lib, name).restype = c_int
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load_library().pi_strerror(code).decode()
+
+
+def _check(call: str, rc: int) -> None:
+    if rc != OK:
+        raise PiError(call, rc, strerror(rc))
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> int:
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def h2d_copy_ms(host_pinned: torch.Tensor, dev: torch.Tensor, reps: int = 10) -> float:
+    """Best time (ms) of a pinned host -> device copy of the whole tensor."""
+    if not host_pinned.is_pinned() or not dev.is_cuda:
+        raise TypeError("h2d_copy_ms: need a pinned host tensor and a CUDA tensor")
+    nbytes = host_pinned.numel() * host_pinned.element_size()
+    assert dev.numel() * dev.element_size() >= nbytes
+    ms = c_float(0)
+    _check("pi_h2d_copy_ms", load_library().pi_h2d_copy_ms(host_pinned.data_ptr(), dev.data_ptr(), nbytes, reps, ctypes.byref(ms)))
+    return float(ms.value)
+
+
+class PulseInfer:
+    """One context = one model shape on the current CUDA device."""
+
+    def __init__(self, *, n_layers: int, n_q_heads: int, n_kv_heads: int, block_tokens: int, budget_blocks: int,
+                 n_sink_blocks: int, n_local_blocks: int, pool_slots: int, max_batch: int, max_blocks: int,
+                 solo_head: Sequence[int], head_dim: int = 128, recall_ctas: int = 0, attn_ctas: int = 0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("paper_2609_34555_b200 needs a CUDA device; there is no CPU path")
+        self._lib = load_library()
+        heads = (c_int32 * n_layers)(*[int(h) for h in solo_head])
+        self.cfg = PiConfig(n_layers, n_q_heads, n_kv_heads, head_dim, block_tokens, budget_blocks, n_sink_blocks,
+                            n_local_blocks, pool_slots, max_batch, max_blocks, recall_ctas, attn_ctas, heads)
+        self._ctx = c_void_p()
+        _check("pi_create", self._lib.pi_create(ctypes.byref(self.cfg), ctypes.byref(self._ctx)))
+        self.frag_bytes = block_tokens * head_dim * 2 * 2
+        self.block_bytes = self.frag_bytes * n_kv_heads
+
+    @classmethod
+    def from_workload(cls, cfg, max_batch: Optional[int] = None, **kw) -> "PulseInfer":
+        return cls(n_layers=cfg.n_layers, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
+                   block_tokens=cfg.block_tokens, budget_blocks=cfg.budget_blocks,
+                   n_sink_blocks=cfg.n_sink_blocks, n_local_blocks=cfg.n_local_blocks, pool_slots=cfg.pool_slots,
+                   max_batch=max_batch or cfg.batch, max_blocks=cfg.n_blocks,
+                   solo_head=[cfg.solo_head(l) for l in range(cfg.n_layers)], head_dim=cfg.head_dim, **kw)
+
+    def close(self) -> None:
+        if getattr(self, "_ctx", None) is not None and self._ctx.value:
+            self._lib.pi_destroy(self._ctx)
+            self._ctx = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ------------------------------------------------------------------ the four path calls
+    def score_select(self, layer: int, q, digest, ctx_len, sel_blocks, sel_count, scores=None, stream=None) -> None:
+        batch = q.shape[0]
+        _check("pi_score_select", self._lib.pi_score_select(
+            self._ctx, layer, batch, _dev(q, torch.bfloat16, "q"), _dev(digest, torch.bfloat16, "digest"),
+            _dev(ctx_len, torch.int32, "ctx_len"), _dev(sel_blocks, torch.int32, "sel_blocks"),
+            _dev(sel_count, torch.int32, "sel_count"),
+            None if scores is None else _dev(scores, torch.float32, "scores"), _stream(stream)))
+
+    def diff_misses(self, layer: int, step: int, ctx_len, sel_blocks, sel_count, block_table, slot_block, slot_stamp,
+                    sel_slots, recall_list, recall_count, stream=None) -> None:
+        batch = sel_count.shape[0]
+        _check("pi_diff_misses", self._lib.pi_diff_misses(
+            self._ctx, layer, batch, step, _dev(ctx_len, torch.int32, "ctx_len"),
+            _dev(sel_blocks, torch.int32, "sel_blocks"), _dev(sel_count, torch.int32, "sel_count"),
+            _dev(block_table, torch.int32, "block_table"), _dev(slot_block, torch.int32, "slot_block"),
+            _dev(slot_stamp, torch.int32, "slot_stamp"), _dev(sel_slots, torch.int32, "sel_slots"),
+            _dev(recall_list, EXTENT_DTYPE, "recall_list"), _dev(recall_count, torch.int32, "recall_count"),
+            _stream(stream)))
+
+    def recall_gather_scatter(self, layer: int, host_kv, pool, recall_list, recall_count, *, lists_per_seq: int = 1,
+                              unit_bytes: Optional[int] = None, host_seq_stride: Optional[int] = None,
+                              pool_seq_stride: Optional[int] = None, stream=None) -> None:
+        """host_kv: pinned host tensor [batch][NB] blocks; pool: CUDA tensor [batch][C] blocks;
+        recall_list: int32 [n_lists][capacity][4]."""
+        n_lists, cap = recall_list.shape[0], recall_list.shape[1]
+        if not host_kv.is_cuda and not host_kv.is_pinned():
+            raise PiError("pi_recall_gather_scatter", -5, strerror(-5))
+        hs = host_seq_stride if host_seq_stride is not None else host_kv.stride(0) * host_kv.element_size()
+        ps = pool_seq_stride if pool_seq_stride is not None else pool.stride(0) * pool.element_size()
+        _check("pi_recall_gather_scatter", self._lib.pi_recall_gather_scatter(
+            self._ctx, layer, n_lists, lists_per_seq, host_kv.data_ptr(), hs, pool.data_ptr(), ps,
+            _dev(recall_list, EXTENT_DTYPE, "recall_list"), cap, _dev(recall_count, torch.int32, "recall_count"),
+            unit_bytes or self.block_bytes, _stream(stream)))
+
+    def sparse_decode_attn(self, layer: int, q, pool, sel_slots, sel_blocks, sel_count, ctx_len, out, lse=None,
+                           stream=None) -> None:
+        batch = q.shape[0]
+        if not pool.is_cuda or not pool.is_contiguous():
+            raise TypeError("pool: expected a contiguous CUDA tensor")
+        _check("pi_sparse_decode_attn", self._lib.pi_sparse_decode_attn(
+            self._ctx, layer, batch, _dev(q, torch.bfloat16, "q"), pool.data_ptr(),
+            _dev(sel_slots, torch.int32, "sel_slots"), _dev(sel_blocks, torch.int32, "sel_blocks"),
+            _dev(sel_count, torch.int32, "sel_count"), _dev(ctx_len, torch.int32, "ctx_len"),
+            _dev(out, torch.bfloat16, "out"), None if lse is None else _dev(lse, torch.float32, "lse"),
+            _stream(stream)))
+
+    # ------------------------------------------------------------------ helpers
+    def build_digests(self, layer: int, kv, ctx_len, digest, kv_seq_stride: Optional[int] = None, stream=None) -> None:
+        batch = ctx_len.shape[0]
+        stride = kv_seq_stride if kv_seq_stride is not None else kv.stride(0) * kv.element_size()
+        _check("pi_build_digests", self._lib.pi_build_digests(
+            self._ctx, layer, batch, kv.data_ptr(), stride, _dev(ctx_len, torch.int32, "ctx_len"),
+            _dev(digest, torch.bfloat16, "digest"), _stream(stream)))
+
+    def table_init(self, resident, block_table, slot_block, slot_stamp, stream=None) -> None:
+        batch = resident.shape[0]
+        _check("pi_table_init", self._lib.pi_table_init(
+            self._ctx, batch, _dev(resident, torch.int32, "resident"), _dev(block_table, torch.int32, "block_table"),
+            _dev(slot_block, torch.int32, "slot_block"), _dev(slot_stamp, torch.int32, "slot_stamp"), _stream(stream)))
+
+    def status(self) -> list[int]:
+        out = (c_int32 * 8)()
+        _check("pi_get_status", self._lib.pi_get_status(self._ctx, ctypes.byref(out)))
+        return list(out)
+
+    def clear_status(self) -> None:
+        _check("pi_clear_status", self._lib.pi_clear_status(self._ctx))

@@ -1,0 +1,267 @@
+// C-ABI entry points: context life cycle, argument checks, status word.
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "pi_common.cuh"
+
+namespace {
+
+bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+
+int check_config(const pi_config* c) {
+    if (!c || !c->solo_head) return PI_ERR_INVALID_ARG;
+    if (c->head_dim != PI_HEAD_DIM) return PI_ERR_UNSUPPORTED_DIM;
+    if (c->block_tokens != 16 && c->block_tokens != 32 && c->block_tokens != 64) return PI_ERR_UNSUPPORTED_DIM;
+    if (c->n_kv_heads < 1 || c->n_kv_heads > 16 || !is_pow2(c->n_kv_heads)) return PI_ERR_UNSUPPORTED_DIM;
+    if (c->n_q_heads < c->n_kv_heads || c->n_q_heads % c->n_kv_heads) return PI_ERR_UNSUPPORTED_DIM;
+    if (c->n_q_heads / c->n_kv_heads > 16) return PI_ERR_UNSUPPORTED_DIM;
+    if (c->n_layers < 1 || c->max_batch < 1 || c->max_batch > 4096) return PI_ERR_INVALID_ARG;
+    if (c->max_blocks < 1 || c->max_blocks > 16384) return PI_ERR_UNSUPPORTED_DIM;
+    if (c->n_sink_blocks < 0 || c->n_local_blocks < 0) return PI_ERR_INVALID_ARG;
+    if (c->budget_blocks < 1 || c->budget_blocks < c->n_sink_blocks + c->n_local_blocks) return PI_ERR_INVALID_ARG;
+    if (c->budget_blocks > 4096) return PI_ERR_UNSUPPORTED_DIM;
+    if (c->pool_slots < c->budget_blocks) return PI_ERR_POOL_TOO_SMALL;
+    if (c->pool_slots > 8192) return PI_ERR_UNSUPPORTED_DIM;
+    if (c->recall_ctas < 0 || c->attn_ctas < 0) return PI_ERR_INVALID_ARG;
+    for (int l = 0; l < c->n_layers; ++l)
+        if (c->solo_head[l] < 0 || c->solo_head[l] >= c->n_kv_heads) return PI_ERR_INVALID_ARG;
+    return PI_OK;
+}
+
+int check_call(pi_ctx* ctx, int layer, int batch) {
+    if (!ctx) return PI_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return PI_ERR_INVALID_ARG;
+    if (batch < 1 || batch > ctx->cfg.max_batch) return PI_ERR_INVALID_ARG;
+    return PI_OK;
+}
+
+}  // namespace
+
+extern "C" int pi_create(const pi_config* cfg, pi_ctx** out) {
+    if (!out) return PI_ERR_INVALID_ARG;
+    *out = nullptr;
+    int rc = check_config(cfg);
+    if (rc != PI_OK) return rc;
+    pi_ctx* c = new (std::nothrow) pi_ctx();
+    if (!c) return PI_ERR_INVALID_ARG;
+    std::memset(c, 0, sizeof(*c));
+    c->cfg = *cfg;
+    c->solo_head = static_cast<int32_t*>(std::malloc(sizeof(int32_t) * cfg->n_layers));
+    std::memcpy(c->solo_head, cfg->solo_head, sizeof(int32_t) * cfg->n_layers);
+    c->cfg.solo_head = c->solo_head;
+
+    cudaError_t e = cudaGetDevice(&c->device);
+    cudaDeviceProp prop;
+    if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, c->device);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); pi_destroy(c); return PI_ERR_CUDA; }
+    c->n_sms = prop.multiProcessorCount;
+    c->attn_ctas = cfg->attn_ctas > 0 ? cfg->attn_ctas : c->n_sms;
+    c->recall_ctas = cfg->recall_ctas > 0 ? cfg->recall_ctas : 32;
+
+    const size_t nb = static_cast<size_t>(cfg->max_batch);
+    const size_t n_part = static_cast<size_t>(c->attn_ctas) + nb;
+    void* host = nullptr;
+    bool ok = cudaMalloc(&c->scores, nb * cfg->max_blocks * sizeof(float)) == cudaSuccess &&
+              cudaMalloc(&c->sel_counters, nb * sizeof(unsigned int)) == cudaSuccess &&
+              cudaMalloc(&c->attn_counters, nb * sizeof(unsigned int)) == cudaSuccess &&
+              cudaMalloc(&c->attn_part_o, n_part * cfg->n_q_heads * PI_HEAD_DIM * sizeof(float)) == cudaSuccess &&
+              cudaMalloc(&c->attn_part_ml, n_part * cfg->n_q_heads * 2 * sizeof(float)) == cudaSuccess &&
+              cudaMalloc(&c->status_flag_dev, sizeof(int)) == cudaSuccess &&
+              cudaHostAlloc(&host, 8 * sizeof(int32_t), cudaHostAllocMapped) == cudaSuccess;
+    if (ok) {
+        c->status_host = static_cast<volatile int32_t*>(host);
+        for (int i = 0; i < 8; ++i) c->status_host[i] = 0;
+        void* alias = nullptr;
+        ok = cudaHostGetDevicePointer(&alias, host, 0) == cudaSuccess &&
+             cudaMemset(c->sel_counters, 0, nb * sizeof(unsigned int)) == cudaSuccess &&
+             cudaMemset(c->attn_counters, 0, nb * sizeof(unsigned int)) == cudaSuccess &&
+             cudaMemset(c->status_flag_dev, 0, sizeof(int)) == cudaSuccess &&
+             cudaDeviceSynchronize() == cudaSuccess;
+        c->status_host_devptr = static_cast<int32_t*>(alias);
+    }
+    if (ok) {
+        cudaDriverEntryPointQueryResult q;
+        ok = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled_fn, cudaEnableDefault, &q) == cudaSuccess &&
+             q == cudaDriverEntryPointSuccess && c->encode_tiled_fn != nullptr;
+    }
+    if (!ok) { (void)cudaGetLastError(); pi_destroy(c); return PI_ERR_CUDA; }
+    *out = c;
+    return PI_OK;
+}
+
+extern "C" int pi_destroy(pi_ctx* c) {
+    if (!c) return PI_ERR_INVALID_ARG;
+    cudaFree(c->scores);
+    cudaFree(c->sel_counters);
+    cudaFree(c->attn_counters);
+    cudaFree(c->attn_part_o);
+    cudaFree(c->attn_part_ml);
+    cudaFree(c->status_flag_dev);
+    if (c->status_host) cudaFreeHost(const_cast<int32_t*>(c->status_host));
+    (void)cudaGetLastError();
+    std::free(c->solo_head);
+    delete c;
+    return PI_OK;
+}
+
+extern "C" int pi_score_select(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* digest_dev,
+                               const int32_t* ctx_len_dev, int32_t* sel_blocks_dev, int32_t* sel_count_dev,
+                               float* scores_dev, void* stream) {
+    int rc = check_call(ctx, layer, batch);
+    if (rc != PI_OK) return rc;
+    if (!q_dev || !digest_dev || !ctx_len_dev || !sel_blocks_dev || !sel_count_dev) return PI_ERR_INVALID_ARG;
+    if (!pi_aligned16(q_dev) || !pi_aligned16(digest_dev)) return PI_ERR_BAD_ALIGN;
+    return pi_launch_score_select(ctx, ctx->solo_head[layer], batch, q_dev, digest_dev, ctx_len_dev,
+                                  sel_blocks_dev, sel_count_dev, scores_dev ? scores_dev : ctx->scores,
+                                  ctx->sel_counters, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int pi_diff_misses(pi_ctx* ctx, int layer, int batch, uint32_t step, const int32_t* ctx_len_dev,
+                              const int32_t* sel_blocks_dev, const int32_t* sel_count_dev,
+                              int32_t* block_table_dev, int32_t* slot_block_dev, uint32_t* slot_stamp_dev,
+                              int32_t* sel_slots_dev, pi_extent* recall_list_dev, int32_t* recall_count_dev,
+                              void* stream) {
+    int rc = check_call(ctx, layer, batch);
+    if (rc != PI_OK) return rc;
+    if (!ctx_len_dev || !sel_blocks_dev || !sel_count_dev || !block_table_dev || !slot_block_dev ||
+        !slot_stamp_dev || !sel_slots_dev || !recall_list_dev || !recall_count_dev || step == 0)
+        return PI_ERR_INVALID_ARG;
+    if (!pi_aligned16(recall_list_dev)) return PI_ERR_BAD_ALIGN;
+    return pi_launch_diff(ctx, batch, step, ctx_len_dev, sel_blocks_dev, sel_count_dev, block_table_dev,
+                          slot_block_dev, slot_stamp_dev, sel_slots_dev, recall_list_dev, recall_count_dev,
+                          static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int pi_recall_gather_scatter(pi_ctx* ctx, int layer, int n_lists, int lists_per_seq,
+                                        const void* host_kv_pinned, int64_t host_seq_stride_bytes,
+                                        void* pool_dev, int64_t pool_seq_stride_bytes,
+                                        const pi_extent* recall_list_dev, int32_t list_capacity,
+                                        const int32_t* recall_count_dev, int64_t unit_bytes, void* stream) {
+    if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers) return PI_ERR_INVALID_ARG;
+    if (n_lists < 1 || lists_per_seq < 1 || n_lists % lists_per_seq || n_lists > 65536) return PI_ERR_INVALID_ARG;
+    if (!host_kv_pinned || !pool_dev || !recall_list_dev || !recall_count_dev || list_capacity < 1)
+        return PI_ERR_INVALID_ARG;
+    if (unit_bytes < 4096 || unit_bytes % 4096 || unit_bytes > (1 << 24)) return PI_ERR_UNSUPPORTED_DIM;
+    if (host_seq_stride_bytes % 16 || pool_seq_stride_bytes % 16 || host_seq_stride_bytes < 0 ||
+        pool_seq_stride_bytes < 0)
+        return PI_ERR_BAD_ALIGN;
+    if (!pi_aligned16(host_kv_pinned) || !pi_aligned16(pool_dev) || !pi_aligned16(recall_list_dev))
+        return PI_ERR_BAD_ALIGN;
+    // the store must be memory the GPU can address: pinned host (or device) memory
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, host_kv_pinned) != cudaSuccess) { (void)cudaGetLastError(); return PI_ERR_NOT_PINNED; }
+    const void* src = host_kv_pinned;
+    if (attr.type == cudaMemoryTypeHost) {
+        if (!attr.devicePointer) return PI_ERR_NOT_PINNED;
+        src = attr.devicePointer;
+    } else if (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged) {
+        return PI_ERR_NOT_PINNED;
+    }
+    return pi_launch_recall(ctx, n_lists, lists_per_seq, src, host_seq_stride_bytes, pool_dev,
+                            pool_seq_stride_bytes, recall_list_dev, list_capacity, recall_count_dev,
+                            unit_bytes, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int pi_sparse_decode_attn(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* pool_dev,
+                                     const int32_t* sel_slots_dev, const int32_t* sel_blocks_dev,
+                                     const int32_t* sel_count_dev, const int32_t* ctx_len_dev, void* out_dev,
+                                     float* lse_dev, void* stream) {
+    int rc = check_call(ctx, layer, batch);
+    if (rc != PI_OK) return rc;
+    if (!q_dev || !pool_dev || !sel_slots_dev || !sel_blocks_dev || !sel_count_dev || !ctx_len_dev || !out_dev)
+        return PI_ERR_INVALID_ARG;
+    if (!pi_aligned16(q_dev) || !pi_aligned16(out_dev) || (reinterpret_cast<uintptr_t>(pool_dev) & 127u))
+        return PI_ERR_BAD_ALIGN;
+    return pi_launch_attn(ctx, batch, q_dev, pool_dev, sel_slots_dev, sel_blocks_dev, sel_count_dev,
+                          ctx_len_dev, out_dev, lse_dev, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int pi_build_digests(pi_ctx* ctx, int layer, int batch, const void* kv, int64_t kv_seq_stride_bytes,
+                                const int32_t* ctx_len_dev, void* digest_dev, void* stream) {
+    int rc = check_call(ctx, layer, batch);
+    if (rc != PI_OK) return rc;
+    if (!kv || !ctx_len_dev || !digest_dev || kv_seq_stride_bytes < 0) return PI_ERR_INVALID_ARG;
+    if (!pi_aligned16(kv) || !pi_aligned16(digest_dev) || kv_seq_stride_bytes % 16) return PI_ERR_BAD_ALIGN;
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, kv) != cudaSuccess) { (void)cudaGetLastError(); return PI_ERR_NOT_PINNED; }
+    const void* src = kv;
+    if (attr.type == cudaMemoryTypeHost) {
+        if (!attr.devicePointer) return PI_ERR_NOT_PINNED;
+        src = attr.devicePointer;
+    } else if (attr.type == cudaMemoryTypeUnregistered) {
+        return PI_ERR_NOT_PINNED;
+    }
+    return pi_launch_build_digests(ctx, ctx->solo_head[layer], batch, src, kv_seq_stride_bytes, ctx_len_dev,
+                                   digest_dev, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int pi_table_init(pi_ctx* ctx, int batch, const int32_t* resident_dev, int32_t* block_table_dev,
+                             int32_t* slot_block_dev, uint32_t* slot_stamp_dev, void* stream) {
+    int rc = check_call(ctx, 0, batch);
+    if (rc != PI_OK) return rc;
+    if (!resident_dev || !block_table_dev || !slot_block_dev || !slot_stamp_dev) return PI_ERR_INVALID_ARG;
+    return pi_launch_table_init(ctx, batch, resident_dev, block_table_dev, slot_block_dev, slot_stamp_dev,
+                                static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int pi_h2d_copy_ms(const void* host_pinned, void* dev, int64_t bytes, int reps, float* best_ms) {
+    if (!host_pinned || !dev || bytes <= 0 || reps < 1 || !best_ms) return PI_ERR_INVALID_ARG;
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, host_pinned) != cudaSuccess || attr.type != cudaMemoryTypeHost) {
+        (void)cudaGetLastError();
+        return PI_ERR_NOT_PINNED;
+    }
+    cudaEvent_t a, b;
+    PI_CUDA_TRY(cudaEventCreate(&a));
+    PI_CUDA_TRY(cudaEventCreate(&b));
+    float best = 1e30f;
+    int rc = PI_OK;
+    for (int i = 0; i < reps + 1 && rc == PI_OK; ++i) {   // first copy is a warm-up
+        float ms = 0.f;
+        if (cudaEventRecord(a, 0) != cudaSuccess ||
+            cudaMemcpyAsync(dev, host_pinned, static_cast<size_t>(bytes), cudaMemcpyHostToDevice, 0) != cudaSuccess ||
+            cudaEventRecord(b, 0) != cudaSuccess || cudaEventSynchronize(b) != cudaSuccess ||
+            cudaEventElapsedTime(&ms, a, b) != cudaSuccess) {
+            (void)cudaGetLastError();
+            rc = PI_ERR_CUDA;
+        } else if (i > 0 && ms < best) {
+            best = ms;
+        }
+    }
+    cudaEventDestroy(a);
+    cudaEventDestroy(b);
+    *best_ms = best;
+    return rc;
+}
+
+extern "C" int pi_get_status(pi_ctx* ctx, int32_t out[8]) {
+    if (!ctx || !out) return PI_ERR_INVALID_ARG;
+    for (int i = 0; i < 8; ++i) out[i] = ctx->status_host[i];
+    return PI_OK;
+}
+
+extern "C" int pi_clear_status(pi_ctx* ctx) {
+    if (!ctx) return PI_ERR_INVALID_ARG;
+    PI_CUDA_TRY(cudaDeviceSynchronize());
+    PI_CUDA_TRY(cudaMemset(ctx->status_flag_dev, 0, sizeof(int)));
+    for (int i = 0; i < 8; ++i) ctx->status_host[i] = 0;
+    PI_CUDA_TRY(cudaDeviceSynchronize());
+    return PI_OK;
+}
+
+extern "C" const char* pi_strerror(int code) {
+    switch (code) {
+        case PI_OK: return "ok";
+        case PI_ERR_INVALID_ARG: return "invalid argument";
+        case PI_ERR_BAD_ALIGN: return "pointer or stride not 16-byte aligned";
+        case PI_ERR_UNSUPPORTED_DIM: return "unsupported dimension";
+        case PI_ERR_POOL_TOO_SMALL: return "pool has too few evictable slots";
+        case PI_ERR_NOT_PINNED: return "host store is not GPU-addressable (pin it)";
+        case PI_ERR_CUDA: return "CUDA runtime error";
+        case PI_ERR_TIMEOUT: return "bounded device wait ran out";
+        case PI_ERR_INDEX_RANGE: return "index read from a device list is out of range";
+        case PI_ERR_CAPACITY: return "count read from device memory exceeds capacity";
+        default: return "unknown error";
+    }
+}

@@ -1,0 +1,476 @@
+// Sparse GQA decode attention over the selected pool slots.
+//
+// Work is one flat list of "units": (sequence, selected block, 16-token sub-tile),
+// each unit being the K and V rows of those 16 tokens for ALL kv heads (Hkv * 8 KB).
+// A persistent grid splits the list evenly (split-K across CTAs, ranges may cross
+// sequence boundaries); a CTA is one TMA producer warp plus one consumer warp per kv
+// head.  The producer streams units through a ring of shared-memory stages with
+// tiled TMA loads (128-byte swizzle, no multicast); consumer warp h computes, for its
+// G query heads,  S^T = K q^T  (tokens on M, heads on N, bf16 mma, fp32 accumulate),
+// an online softmax over tokens, and  O^T += V^T P.  A (CTA, sequence) segment that
+// does not cover its whole sequence writes an fp32 partial (m, l, O); the CTA whose
+// ticket completes the sequence merges the partials.  No CTA waits for another.
+//
+// The arithmetic intensity is G flop per byte: HBM-bound by a wide margin, so the
+// design goal is bytes in flight (ring of Hkv*8 KB stages), not tensor throughput.
+#include "pi_common.cuh"
+
+namespace {
+
+constexpr int ATTN_MAX_STAGES = 8;
+constexpr int ATTN_META_UNITS = 1024;              // units per CTA whose metadata is staged in shared memory
+constexpr int ATTN_SMEM_BUDGET = 196 * 1024;       // ring bytes
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s: a wait this long is a failure
+
+struct AttnParams {
+    const __nv_bfloat16* q;
+    const int32_t* sel_slots;
+    const int32_t* sel_blocks;
+    const int32_t* sel_count;
+    const int32_t* ctx_len;
+    __nv_bfloat16* out;
+    float* lse;
+    float* part_o;
+    float* part_ml;
+    unsigned int* counters;
+    pi_status_ref st;
+    int batch, Hq, Hkv, G, B, K, C, stages;
+    float scale_log2;
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up when another warp raised `abort` or the cycle limit passes.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try(bar, parity)) return true;
+        if (*abort) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort = 1; return false; }
+    }
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ uint32_t movm_t(uint32_t x) {
+    uint32_t y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+    return y;
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// CTA that owns unit u when U units are split over P CTAs as [U*c/P, U*(c+1)/P).
+__device__ __forceinline__ int cta_of_unit(long long u, long long U, long long P) {
+    long long c = (u * P) / U;
+    while ((U * (c + 1)) / P <= u) ++c;
+    while ((U * c) / P > u) --c;
+    return static_cast<int>(c);
+}
+
+__device__ __forceinline__ int seq_of_unit(const int* pref, int batch, int u) {
+    int lo = 0, hi = batch;                          // last s with pref[s] <= u
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (pref[mid] <= u) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+template <int NT>
+__global__ void __launch_bounds__(288, 1)
+attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
+    extern __shared__ unsigned char smem_dyn[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int stage_bytes = p.Hkv * 8192, half_bytes = p.Hkv * 4096;
+    const uint32_t ring = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    unsigned char* after_ring = smem_dyn + (ring - smem_u32(smem_dyn)) + static_cast<size_t>(p.stages) * stage_bytes;
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(after_ring);      // full[8], empty[8], seg
+    int* s_nvalid = reinterpret_cast<int*>(bars + 2 * ATTN_MAX_STAGES + 1);            // [8]
+    int* s_abort = s_nvalid + ATTN_MAX_STAGES;
+    int* s_last = s_abort + 1;
+    int2* s_meta = reinterpret_cast<int2*>(s_last + 1);                                // [ATTN_META_UNITS] {slot row, sub*16 | nvalid<<8}
+    int* s_pref = reinterpret_cast<int*>(s_meta + ATTN_META_UNITS);                    // [batch + 1]
+    const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + ATTN_MAX_STAGES);
+    const uint32_t bar_seg = smem_u32(bars + 2 * ATTN_MAX_STAGES);
+    const int SUB = p.B >> 4;
+
+    // ---- unit prefix over sequences (every CTA computes the same table)
+    for (int s = tid; s < p.batch; s += blockDim.x) {
+        int n = p.sel_count[s];
+        if (n < 0 || n > p.K) {
+            if (blockIdx.x == 0) pi_report(p.st, PI_ERR_CAPACITY, PI_STAGE_ATTN, s, n, p.K);
+            n = 0;
+        }
+        s_pref[s + 1] = n * SUB;
+    }
+    if (tid == 0) {
+        s_pref[0] = 0;
+        *s_abort = 0;
+        for (int i = 0; i < p.stages; ++i) {
+            mbar_init(bar_full + 8 * i, 1);
+            mbar_init(bar_empty + 8 * i, p.Hkv);
+        }
+        mbar_init(bar_seg, p.Hkv);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 0) {                                   // inclusive scan in place, 32 entries a time
+        int run = 0;
+        for (int s0 = 0; s0 < p.batch; s0 += 32) {
+            const int s = s0 + lane;
+            int v = s < p.batch ? s_pref[s + 1] : 0;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                int t = __shfl_up_sync(0xffffffffu, v, o);
+                if (lane >= o) v += t;
+            }
+            if (s < p.batch) s_pref[s + 1] = run + v;
+            run += __shfl_sync(0xffffffffu, v, 31);
+        }
+    }
+    __syncthreads();
+
+    // never more CTAs than units: then every CTA in [0, P) owns at least one unit, which the
+    // segment count of a sequence (last owner - first owner + 1) relies on
+    const long long U = s_pref[p.batch], P = min(static_cast<long long>(gridDim.x), max(U, 1ll));
+    // sequences with nothing selected: defined output, written by CTA 0
+    if (blockIdx.x == 0) {
+        for (int s = 0; s < p.batch; ++s) {
+            if (s_pref[s + 1] != s_pref[s]) continue;
+            for (int i = tid; i < p.Hq * PI_HEAD_DIM; i += blockDim.x)
+                p.out[static_cast<size_t>(s) * p.Hq * PI_HEAD_DIM + i] = __float2bfloat16(0.f);
+            if (p.lse)
+                for (int i = tid; i < p.Hq; i += blockDim.x) p.lse[static_cast<size_t>(s) * p.Hq + i] = -INFINITY;
+        }
+    }
+    if (U == 0 || blockIdx.x >= P) return;
+    const int u0 = static_cast<int>((U * blockIdx.x) / P), u1 = static_cast<int>((U * (blockIdx.x + 1)) / P);
+    if (u0 >= u1) return;
+
+    // ---- metadata of this CTA's units: global row of the slot, token offset, valid tokens.
+    // Staged up front by all threads so the producer never waits on a dependent global load.
+    auto unit_meta = [&](int u, int seq) -> int2 {
+        const int r = u - s_pref[seq], j = r / SUB, sub = r - j * SUB;
+        int slot = p.sel_slots[static_cast<size_t>(seq) * p.K + j];
+        const int blk = p.sel_blocks[static_cast<size_t>(seq) * p.K + j];
+        if (slot < 0 || slot >= p.C) {
+            pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_ATTN, seq, j, slot);
+            slot = 0;
+        }
+        const int nvalid = blk < 0 ? 0 : max(0, min(16, p.ctx_len[seq] - (blk * p.B + sub * 16)));
+        return make_int2(seq * p.C + slot, (sub * 16) | (nvalid << 8));
+    };
+    for (int i = tid; i < u1 - u0 && i < ATTN_META_UNITS; i += blockDim.x)
+        s_meta[i] = unit_meta(u0 + i, seq_of_unit(s_pref, p.batch, u0 + i));
+    __syncthreads();
+
+    if (warp == p.Hkv) {
+        // =============================== producer: one lane issues all TMA loads
+        if (lane == 0) {
+            int seq = seq_of_unit(s_pref, p.batch, u0);
+            for (int u = u0, it = 0; u < u1; ++u, ++it) {
+                while (u >= s_pref[seq + 1]) ++seq;
+                const int2 md = it < ATTN_META_UNITS ? s_meta[it] : unit_meta(u, seq);
+                const int st = it % p.stages, round = it / p.stages;
+                if (round > 0 && !mbar_wait(bar_empty + 8 * st, (round - 1) & 1, s_abort)) break;
+                s_nvalid[st] = md.y >> 8;
+                const uint32_t dst = ring + st * stage_bytes;
+                mbar_expect_tx(bar_full + 8 * st, stage_bytes);
+                tma_load_4d(dst, &pool_map, bar_full + 8 * st, 0, md.y & 0xff, 0, md.x);
+                tma_load_4d(dst + half_bytes, &pool_map, bar_full + 8 * st, 64, md.y & 0xff, 0, md.x);
+            }
+        }
+        return;
+    }
+    if (warp > p.Hkv) return;
+
+    // =============================== consumers: warp h owns kv head h
+    const int h = warp;
+    const int row = lane >> 2, colp = (lane & 3) * 2;
+    uint32_t bq[NT][8][2];
+    float o[NT][8][4], m[NT][2], l[NT][2];
+    int seq = seq_of_unit(s_pref, p.batch, u0);
+    bool fresh = true;
+    int seg_round = 0;
+    // per-lane ldmatrix offsets inside a stage (swizzled 128-byte rows)
+    const int r8 = lane & 7, mi = lane >> 3;
+    const int tK = r8 + 8 * (mi & 1), cK = mi >> 1;         // K as A operand (rows = tokens)
+    const int tV = r8 + 8 * (mi >> 1), cV = mi & 1;         // V^T as A operand via .trans
+    const uint32_t offK = (2 * h) * 2048 + tK * 128, offV = (2 * h + 1) * 2048 + tV * 128;
+
+    for (int u = u0, it = 0; u < u1; ++u, ++it) {
+        while (u >= s_pref[seq + 1]) { ++seq; fresh = true; }
+        if (fresh) {
+            fresh = false;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                const int g = nt * 8 + row;
+                const __nv_bfloat16* qg = p.q + (static_cast<size_t>(seq) * p.Hq + static_cast<size_t>(h) * p.G + g) * PI_HEAD_DIM + colp;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    bq[nt][j][0] = g < p.G ? *reinterpret_cast<const uint32_t*>(qg + 16 * j) : 0u;
+                    bq[nt][j][1] = g < p.G ? *reinterpret_cast<const uint32_t*>(qg + 16 * j + 8) : 0u;
+                }
+                m[nt][0] = m[nt][1] = -INFINITY;
+                l[nt][0] = l[nt][1] = 0.f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) o[nt][i][0] = o[nt][i][1] = o[nt][i][2] = o[nt][i][3] = 0.f;
+            }
+        }
+        const int st = it % p.stages;
+        if (!mbar_wait(bar_full + 8 * st, (it / p.stages) & 1, s_abort)) break;
+        const int nvalid = s_nvalid[st];
+        const uint32_t base = ring + st * stage_bytes;
+
+        // ---- S^T = K q^T
+        float c[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            uint32_t a[4];
+            const int chunk = 2 * (j & 3) + cK;
+            ldsm_x4(base + (j >> 2) * half_bytes + offK + ((chunk ^ r8) << 4), a);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) mma_bf16(c[nt], a, bq[nt][j][0], bq[nt][j][1]);
+        }
+        // ---- online softmax over tokens (rows), one state per query head (column)
+        // P is split into a bf16 head and a bf16 remainder (two MMAs per V tile): value
+        // channels with large magnitudes would otherwise see the 2^-9 rounding of P directly.
+        uint32_t pb[NT][2], pl[NT][2];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            float pr[4];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                float s0 = row < nvalid ? c[nt][e] * p.scale_log2 : -INFINITY;
+                float s1 = row + 8 < nvalid ? c[nt][e + 2] * p.scale_log2 : -INFINITY;
+                float mx = fmaxf(s0, s1);
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+                const float m_new = fmaxf(m[nt][e], mx);
+                float alpha = 1.f, p0 = 0.f, p1 = 0.f;
+                if (m_new != -INFINITY) {
+                    alpha = exp2f(m[nt][e] - m_new);
+                    p0 = exp2f(s0 - m_new);
+                    p1 = exp2f(s1 - m_new);
+                }
+                m[nt][e] = m_new;
+                l[nt][e] = l[nt][e] * alpha + p0 + p1;
+                pr[e] = p0; pr[e + 2] = p1;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { o[nt][i][e] *= alpha; o[nt][i][e + 2] *= alpha; }
+            }
+            // P^T fragments (rows = tokens) -> B operand (k = tokens, n = heads)
+            const uint32_t h01 = pack_bf16(pr[0], pr[1]), h23 = pack_bf16(pr[2], pr[3]);
+            const float2 f01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&h01));
+            const float2 f23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&h23));
+            pb[nt][0] = movm_t(h01);
+            pb[nt][1] = movm_t(h23);
+            pl[nt][0] = movm_t(pack_bf16(pr[0] - f01.x, pr[1] - f01.y));
+            pl[nt][1] = movm_t(pack_bf16(pr[2] - f23.x, pr[3] - f23.y));
+        }
+        // ---- O^T += V^T P
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            uint32_t a[4];
+            const int chunk = 2 * (i & 3) + cV;
+            ldsm_x4_t(base + (i >> 2) * half_bytes + offV + ((chunk ^ r8) << 4), a);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                mma_bf16(o[nt][i], a, pb[nt][0], pb[nt][1]);
+                mma_bf16(o[nt][i], a, pl[nt][0], pl[nt][1]);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_empty + 8 * st);
+
+        // ---- end of this CTA's segment of the sequence?
+        if (u + 1 == u1 || u + 1 == s_pref[seq + 1]) {
+            const int c_first = cta_of_unit(s_pref[seq], U, P), c_last = cta_of_unit(s_pref[seq + 1] - 1, U, P);
+            const int n_seg = c_last - c_first + 1;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    float v = l[nt][e];
+                    v += __shfl_xor_sync(0xffffffffu, v, 4);
+                    v += __shfl_xor_sync(0xffffffffu, v, 8);
+                    v += __shfl_xor_sync(0xffffffffu, v, 16);
+                    l[nt][e] = v;
+                }
+            if (n_seg == 1) {
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int g = nt * 8 + colp + e;
+                        if (g >= p.G) continue;
+                        const size_t gh = static_cast<size_t>(seq) * p.Hq + static_cast<size_t>(h) * p.G + g;
+                        const float inv = l[nt][e] > 0.f ? 1.f / l[nt][e] : 0.f;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            p.out[gh * PI_HEAD_DIM + 16 * i + row] = __float2bfloat16(o[nt][i][e] * inv);
+                            p.out[gh * PI_HEAD_DIM + 16 * i + row + 8] = __float2bfloat16(o[nt][i][e + 2] * inv);
+                        }
+                        if (p.lse && row == 0)
+                            p.lse[gh] = l[nt][e] > 0.f ? (m[nt][e] + log2f(l[nt][e])) * 0.6931471805599453f : -INFINITY;
+                    }
+            } else {
+                const size_t pslot = static_cast<size_t>(blockIdx.x) + seq;
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int g = nt * 8 + colp + e;
+                        if (g >= p.G) continue;
+                        const size_t gh = pslot * p.Hq + static_cast<size_t>(h) * p.G + g;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            p.part_o[gh * PI_HEAD_DIM + 16 * i + row] = o[nt][i][e];
+                            p.part_o[gh * PI_HEAD_DIM + 16 * i + row + 8] = o[nt][i][e + 2];
+                        }
+                        if (row == 0) { p.part_ml[gh * 2] = m[nt][e]; p.part_ml[gh * 2 + 1] = l[nt][e]; }
+                    }
+                __threadfence();
+                __syncwarp();
+                // all consumer warps have published their partials -> one ticket for the CTA
+                if (lane == 0) mbar_arrive(bar_seg);
+                if (!mbar_wait(bar_seg, seg_round & 1, s_abort)) break;
+                if (warp == 0 && lane == 0) {
+                    const unsigned t = atomicAdd(&p.counters[seq], 1u);
+                    const int last = (t == static_cast<unsigned>(n_seg - 1));
+                    if (last) p.counters[seq] = 0;
+                    *s_last = last;
+                }
+                if (lane == 0) mbar_arrive(bar_seg);
+                if (!mbar_wait(bar_seg, (seg_round + 1) & 1, s_abort)) break;
+                seg_round += 2;
+                if (*s_last) {
+                    __threadfence();
+                    // merge: warp h reduces its G heads over the n_seg partials; lane owns 4 channels
+                    for (int g = 0; g < p.G; ++g) {
+                        const size_t head = static_cast<size_t>(h) * p.G + g;
+                        float M = -INFINITY;
+                        for (int cc = c_first; cc <= c_last; ++cc)
+                            M = fmaxf(M, __ldcg(p.part_ml + ((static_cast<size_t>(cc) + seq) * p.Hq + head) * 2));
+                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                        float L = 0.f;
+                        for (int cc = c_first; cc <= c_last; ++cc) {
+                            const size_t gh = (static_cast<size_t>(cc) + seq) * p.Hq + head;
+                            const float mi_ = __ldcg(p.part_ml + gh * 2), li_ = __ldcg(p.part_ml + gh * 2 + 1);
+                            const float w = (mi_ == -INFINITY) ? 0.f : exp2f(mi_ - M);
+                            const float4 v = __ldcg(reinterpret_cast<const float4*>(p.part_o + gh * PI_HEAD_DIM) + lane);
+                            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+                            L += w * li_;
+                        }
+                        const float inv = L > 0.f ? 1.f / L : 0.f;
+                        const size_t go = (static_cast<size_t>(seq) * p.Hq + head) * PI_HEAD_DIM + lane * 4;
+                        __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+                        __nv_bfloat162 hi2 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+                        uint2 pk;
+                        pk.x = *reinterpret_cast<uint32_t*>(&lo2);
+                        pk.y = *reinterpret_cast<uint32_t*>(&hi2);
+                        *reinterpret_cast<uint2*>(p.out + go) = pk;
+                        if (p.lse && lane == 0)
+                            p.lse[static_cast<size_t>(seq) * p.Hq + head] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
+                    }
+                }
+                // the flag is rewritten only after every warp passed the next pair of barriers
+            }
+        }
+    }
+    if (*s_abort && lane == 0 && warp == 0) pi_report(p.st, PI_ERR_TIMEOUT, PI_STAGE_ATTN, blockIdx.x, u0, u1);
+}
+
+}  // namespace
+
+int pi_launch_attn(pi_ctx* c, int batch, const void* q, const void* pool, const int32_t* sel_slots,
+                   const int32_t* sel_blocks, const int32_t* sel_count, const int32_t* ctx_len, void* out,
+                   float* lse, cudaStream_t stream) {
+    const pi_config& cfg = c->cfg;
+    if (cfg.n_kv_heads > 8) return PI_ERR_UNSUPPORTED_DIM;
+    const long long n_slots = static_cast<long long>(batch) * cfg.pool_slots;
+    if (c->pool_map_ptr != pool || c->pool_map_slots != n_slots) {
+        typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+        const cuuint64_t B = cfg.block_tokens, hk = 2ull * cfg.n_kv_heads;
+        cuuint64_t gdim[4] = {PI_HEAD_DIM, B, hk, static_cast<cuuint64_t>(n_slots)};
+        cuuint64_t gstride[3] = {PI_HEAD_DIM * 2ull, B * PI_HEAD_DIM * 2ull, hk * B * PI_HEAD_DIM * 2ull};
+        cuuint32_t box[4] = {64, 16, static_cast<cuuint32_t>(hk), 1};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        CUresult r = reinterpret_cast<encode_fn>(c->encode_tiled_fn)(
+            &c->pool_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), gdim, gstride, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) { c->pool_map_ptr = nullptr; return PI_ERR_CUDA; }
+        c->pool_map_ptr = pool;
+        c->pool_map_slots = n_slots;
+    }
+    AttnParams p;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.sel_slots = sel_slots; p.sel_blocks = sel_blocks; p.sel_count = sel_count; p.ctx_len = ctx_len;
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.lse = lse;
+    p.part_o = c->attn_part_o; p.part_ml = c->attn_part_ml; p.counters = c->attn_counters;
+    p.st = pi_status_of(c);
+    p.batch = batch; p.Hq = cfg.n_q_heads; p.Hkv = cfg.n_kv_heads; p.G = cfg.n_q_heads / cfg.n_kv_heads;
+    p.B = cfg.block_tokens; p.K = cfg.budget_blocks; p.C = cfg.pool_slots;
+    const int stage_bytes = cfg.n_kv_heads * 8192;
+    int stages = ATTN_SMEM_BUDGET / stage_bytes;
+    if (stages > ATTN_MAX_STAGES) stages = ATTN_MAX_STAGES;
+    p.stages = stages;
+    p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(PI_HEAD_DIM));
+    const size_t smem = 1024 + static_cast<size_t>(stages) * stage_bytes + (2 * ATTN_MAX_STAGES + 1) * 8 +
+                        (ATTN_MAX_STAGES + 2) * 4 + ATTN_META_UNITS * 8 + (static_cast<size_t>(batch) + 1) * 4 + 16;
+    const int threads = (cfg.n_kv_heads + 1) * 32;
+    if (p.G <= 8) {
+        PI_CUDA_TRY(cudaFuncSetAttribute(attn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+        attn_kernel<1><<<c->attn_ctas, threads, smem, stream>>>(c->pool_map, p);
+    } else {
+        PI_CUDA_TRY(cudaFuncSetAttribute(attn_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+        attn_kernel<2><<<c->attn_ctas, threads, smem, stream>>>(c->pool_map, p);
+    }
+    PI_CUDA_TRY(cudaGetLastError());
+    return PI_OK;
+}

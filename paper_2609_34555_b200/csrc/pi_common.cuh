@@ -1,0 +1,89 @@
+// Shared declarations of the CUDA library: context, status word, small device helpers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda.h>
+#include <stdint.h>
+
+#include "pulseinfer.h"
+
+#define PI_STAGE_SELECT 1
+#define PI_STAGE_DIFF   2
+#define PI_STAGE_RECALL 3
+#define PI_STAGE_ATTN   4
+
+#define PI_HEAD_DIM 128
+#define PI_SELECT_BINS 2048
+
+struct pi_ctx {
+    pi_config cfg;
+    int32_t* solo_head;          // host copy [n_layers]
+    int device;
+    int n_sms;
+    // device scratch
+    float* scores;               // [max_batch][max_blocks]
+    unsigned int* sel_counters;  // [max_batch], zero between launches
+    unsigned int* attn_counters; // [max_batch], zero between launches
+    float* attn_part_o;          // [attn_ctas + max_batch][Hq][D]
+    float* attn_part_ml;         // [attn_ctas + max_batch][Hq][2]
+    int attn_ctas, recall_ctas;
+    // status: device flag (first writer wins) + pinned mirror the kernels fill in
+    int* status_flag_dev;
+    volatile int32_t* status_host;   // pinned, 8 ints
+    int32_t* status_host_devptr;     // device alias of status_host
+    // cached tensor map of the pool for the attention kernel
+    CUtensorMap pool_map;
+    const void* pool_map_ptr;
+    long long pool_map_slots;
+    void* encode_tiled_fn;
+};
+
+struct pi_status_ref {
+    int* flag;
+    int32_t* mirror;
+};
+
+__device__ __forceinline__ void pi_report(pi_status_ref st, int code, int stage, int a, int b, int c) {
+    if (atomicCAS(st.flag, 0, code) == 0) {
+        volatile int32_t* m = st.mirror;
+        m[1] = stage; m[2] = a; m[3] = b; m[4] = c;
+        __threadfence_system();
+        m[0] = code;
+    }
+}
+
+static inline pi_status_ref pi_status_of(pi_ctx* c) {
+    pi_status_ref r;
+    r.flag = c->status_flag_dev;
+    r.mirror = c->status_host_devptr;
+    return r;
+}
+
+#define PI_CUDA_TRY(expr)                                  \
+    do {                                                   \
+        cudaError_t e__ = (expr);                          \
+        if (e__ != cudaSuccess) { (void)cudaGetLastError(); return PI_ERR_CUDA; } \
+    } while (0)
+
+static inline bool pi_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+__device__ __forceinline__ int pi_ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Launchers implemented one per .cu file.
+int pi_launch_score_select(pi_ctx*, int h_star, int batch, const void* q, const void* digest,
+                           const int32_t* ctx_len, int32_t* sel, int32_t* sel_count, float* scores,
+                           unsigned int* counters, cudaStream_t);
+int pi_launch_diff(pi_ctx*, int batch, uint32_t step, const int32_t* ctx_len, const int32_t* sel,
+                   const int32_t* sel_count, int32_t* table, int32_t* slot_block, uint32_t* slot_stamp,
+                   int32_t* sel_slots, pi_extent* list, int32_t* count, cudaStream_t);
+int pi_launch_recall(pi_ctx*, int n_lists, int lists_per_seq, const void* host_kv, int64_t host_stride,
+                     void* pool, int64_t pool_stride, const pi_extent* list, int32_t cap,
+                     const int32_t* count, int64_t unit_bytes, cudaStream_t);
+int pi_launch_attn(pi_ctx*, int batch, const void* q, const void* pool, const int32_t* sel_slots,
+                   const int32_t* sel_blocks, const int32_t* sel_count, const int32_t* ctx_len,
+                   void* out, float* lse, cudaStream_t);
+int pi_launch_build_digests(pi_ctx*, int h_star, int batch, const void* kv, int64_t stride,
+                            const int32_t* ctx_len, void* digest, cudaStream_t);
+int pi_launch_table_init(pi_ctx*, int batch, const int32_t* resident, int32_t* table,
+                         int32_t* slot_block, uint32_t* slot_stamp, cudaStream_t);

@@ -1,0 +1,222 @@
+// Miss diff of the selection against the device-resident block table, victim choice,
+// table update and the coalesced recall list.  One CTA per sequence; everything the
+// sequence needs (selection, slot keys) sits in shared memory.
+//
+//   misses     = selected blocks with block_table[b] < 0, ascending
+//   candidates = slots whose block is neither selected nor sink/local (free slots count),
+//                ordered by (stamp, slot) ascending; the i-th miss takes the i-th candidate
+//   update     = evicted block leaves the table, the miss enters it, every selected
+//                slot gets stamp = step
+//   list       = (block -> slot) pairs, runs that are consecutive on both sides merged
+#include "pi_common.cuh"
+
+namespace {
+
+constexpr int DIFF_THREADS = 256;
+constexpr int DIFF_WARPS = DIFF_THREADS / 32;
+
+struct DiffParams {
+    const int32_t* ctx_len;
+    const int32_t* sel;
+    const int32_t* sel_count;
+    int32_t* table;
+    int32_t* slot_block;
+    uint32_t* slot_stamp;
+    int32_t* sel_slots;
+    pi_extent* list;
+    int32_t* count;
+    pi_status_ref st;
+    uint32_t step;
+    int B, K, C, Cpad, n_sink, n_local, max_blocks;
+};
+
+// Ordered compaction step for up to DIFF_THREADS flags: returns this thread's output
+// position (valid if flag) and adds the round's total to `base` (uniform across the CTA).
+__device__ __forceinline__ int ordered_pos(bool flag, int& base, int* warp_tot) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const unsigned m = __ballot_sync(0xffffffffu, flag);
+    __syncthreads();
+    if (lane == 0) warp_tot[w] = __popc(m);
+    __syncthreads();
+    int off = 0, tot = 0;
+#pragma unroll
+    for (int i = 0; i < DIFF_WARPS; ++i) {
+        const int t = warp_tot[i];
+        if (i < w) off += t;
+        tot += t;
+    }
+    const int pos = base + off + __popc(m & ((1u << lane) - 1u));
+    base += tot;
+    return pos;
+}
+
+__global__ void __launch_bounds__(DIFF_THREADS)
+diff_kernel(DiffParams p) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);       // [Cpad]
+    int32_t* s_sel = reinterpret_cast<int32_t*>(keys + p.Cpad);                         // [K]
+    int32_t* s_slot = s_sel + p.K;                                                      // [K] slot of sel[j]
+    int32_t* s_miss = s_slot + p.K;                                                     // [K] j index of i-th miss
+    unsigned char* s_used = reinterpret_cast<unsigned char*>(s_miss + p.K);             // [C] slot holds a selected block
+    __shared__ int warp_tot[DIFF_WARPS];
+    __shared__ int s_ncand;
+
+    const int seq = blockIdx.x, tid = threadIdx.x;
+    int ctx = p.ctx_len[seq];
+    if (ctx < 0) ctx = 0;
+    const int n_blocks = min((ctx + p.B - 1) / p.B, p.max_blocks);
+    int cnt = p.sel_count[seq];
+    if (cnt < 0 || cnt > p.K) {
+        if (tid == 0) pi_report(p.st, PI_ERR_CAPACITY, PI_STAGE_DIFF, seq, cnt, p.K);
+        cnt = max(0, min(cnt, p.K));
+    }
+    int32_t* table = p.table + static_cast<size_t>(seq) * p.max_blocks;
+    int32_t* slot_block = p.slot_block + static_cast<size_t>(seq) * p.C;
+    uint32_t* slot_stamp = p.slot_stamp + static_cast<size_t>(seq) * p.C;
+    const int32_t* sel = p.sel + static_cast<size_t>(seq) * p.K;
+
+    for (int s = tid; s < p.C; s += DIFF_THREADS) s_used[s] = 0;
+    if (tid == 0) s_ncand = 0;
+    __syncthreads();
+
+    // 1. look the selection up; misses compacted in selection (= ascending block) order
+    int n_miss = 0;
+    for (int j0 = 0; j0 < cnt; j0 += DIFF_THREADS) {
+        const int j = j0 + tid;
+        bool miss = false;
+        if (j < cnt) {
+            int b = sel[j];
+            int slot = -1;
+            if (b < 0 || b >= n_blocks) {
+                pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_DIFF, seq, j, b);
+                b = -1;
+            } else {
+                slot = table[b];
+                if (slot >= p.C) { pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_DIFF, seq, b, slot); slot = -1; b = -1; }
+                else if (slot >= 0) s_used[slot] = 1;
+                else miss = true;
+            }
+            s_sel[j] = b;
+            s_slot[j] = slot;
+        }
+        const int pos = ordered_pos(miss, n_miss, warp_tot);
+        if (miss) s_miss[pos] = j;
+    }
+    __syncthreads();
+
+    // 2. victim candidates keyed by (stamp, slot); everything else sorts to the end
+    int my_cand = 0;
+    for (int s = tid; s < p.Cpad; s += DIFF_THREADS) {
+        unsigned long long key = ~0ull;
+        if (s < p.C && n_miss > 0) {
+            const int b = slot_block[s];
+            const bool pinned = b >= 0 && (b < p.n_sink || b >= n_blocks - p.n_local);
+            if (b < 0 || (!s_used[s] && !pinned)) {
+                key = (static_cast<unsigned long long>(slot_stamp[s]) << 32) | static_cast<unsigned>(s);
+                ++my_cand;
+            }
+        }
+        keys[s] = key;
+    }
+    if (my_cand) atomicAdd(&s_ncand, my_cand);
+    __syncthreads();
+    const bool too_small = s_ncand < n_miss;
+
+    if (n_miss > 0 && !too_small) {
+        // 3. bitonic sort of the candidate keys (ascending)
+        for (int k = 2; k <= p.Cpad; k <<= 1) {
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                for (int i = tid; i < p.Cpad; i += DIFF_THREADS) {
+                    const int l = i ^ j;
+                    if (l > i) {
+                        const unsigned long long a = keys[i], b = keys[l];
+                        const bool up = (i & k) == 0;
+                        if ((a > b) == up) { keys[i] = b; keys[l] = a; }
+                    }
+                }
+                __syncthreads();
+            }
+        }
+        // 4. i-th miss takes the i-th candidate
+        for (int i = tid; i < n_miss; i += DIFF_THREADS) {
+            const int j = s_miss[i];
+            const int slot = static_cast<int>(keys[i] & 0xffffffffull);
+            const int old = slot_block[slot];
+            if (old >= 0 && old < p.max_blocks) table[old] = -1;
+            table[s_sel[j]] = slot;
+            slot_block[slot] = s_sel[j];
+            s_slot[j] = slot;
+        }
+        __syncthreads();
+    } else if (too_small && tid == 0) {
+        pi_report(p.st, PI_ERR_POOL_TOO_SMALL, PI_STAGE_DIFF, seq, n_miss, s_ncand);
+    }
+
+    // 5. stamps and the slot of every selected block
+    int32_t* sel_slots = p.sel_slots + static_cast<size_t>(seq) * p.K;
+    for (int j = tid; j < p.K; j += DIFF_THREADS) {
+        int slot = -1;
+        if (j < cnt) {
+            slot = s_slot[j];
+            if (slot >= 0 && !too_small) slot_stamp[slot] = p.step;
+        }
+        sel_slots[j] = slot;
+    }
+
+    // 6. recall list: heads of runs consecutive in block and in slot
+    pi_extent* list = p.list + static_cast<size_t>(seq) * p.K;
+    int n_ext = 0;
+    if (!too_small) {
+        for (int i0 = 0; i0 < n_miss; i0 += DIFF_THREADS) {
+            const int i = i0 + tid;
+            bool head = false;
+            if (i < n_miss) {
+                const int j = s_miss[i];
+                head = true;
+                if (i > 0) {
+                    const int jp = s_miss[i - 1];
+                    head = !(s_sel[jp] + 1 == s_sel[j] && s_slot[jp] + 1 == s_slot[j]);
+                }
+            }
+            const int pos = ordered_pos(head, n_ext, warp_tot);
+            if (head) {
+                int len = 1;
+                while (i + len < n_miss) {
+                    const int a = s_miss[i + len - 1], b = s_miss[i + len];
+                    if (s_sel[a] + 1 == s_sel[b] && s_slot[a] + 1 == s_slot[b]) ++len; else break;
+                }
+                pi_extent e;
+                e.src_unit = s_sel[s_miss[i]];
+                e.dst_unit = s_slot[s_miss[i]];
+                e.n_units = len;
+                e.units_before = i;
+                list[pos] = e;
+            }
+        }
+    }
+    if (tid == 0) p.count[seq] = n_ext;
+}
+
+}  // namespace
+
+int pi_launch_diff(pi_ctx* c, int batch, uint32_t step, const int32_t* ctx_len, const int32_t* sel,
+                   const int32_t* sel_count, int32_t* table, int32_t* slot_block, uint32_t* slot_stamp,
+                   int32_t* sel_slots, pi_extent* list, int32_t* count, cudaStream_t stream) {
+    DiffParams p;
+    p.ctx_len = ctx_len; p.sel = sel; p.sel_count = sel_count;
+    p.table = table; p.slot_block = slot_block; p.slot_stamp = slot_stamp;
+    p.sel_slots = sel_slots; p.list = list; p.count = count;
+    p.st = pi_status_of(c);
+    p.step = step;
+    p.B = c->cfg.block_tokens; p.K = c->cfg.budget_blocks; p.C = c->cfg.pool_slots;
+    int cpad = 2;
+    while (cpad < p.C) cpad <<= 1;
+    p.Cpad = cpad;
+    p.n_sink = c->cfg.n_sink_blocks; p.n_local = c->cfg.n_local_blocks; p.max_blocks = c->cfg.max_blocks;
+    const size_t smem = static_cast<size_t>(cpad) * 8 + static_cast<size_t>(p.K) * 12 + static_cast<size_t>(p.C);
+    if (smem > 40 * 1024)
+        PI_CUDA_TRY(cudaFuncSetAttribute(diff_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    diff_kernel<<<batch, DIFF_THREADS, smem, stream>>>(p);
+    PI_CUDA_TRY(cudaGetLastError());
+    return PI_OK;
+}

@@ -1,0 +1,65 @@
+// Input-preparation kernels around the path: block digests of the retrieval head and
+// block-table initialisation.  Not hot calls.
+#include "pi_common.cuh"
+
+namespace {
+
+// One thread per (block, channel): min / max of the retrieval head's keys over the
+// block's valid tokens.  The result is one of the inputs, so it is exact in bf16.
+__global__ void build_digests_kernel(const __nv_bfloat16* kv, long long seq_stride_elems, const int32_t* ctx_len,
+                                     __nv_bfloat16* digest, int h_star, int Hkv, int B, int max_blocks) {
+    const int seq = blockIdx.y;
+    const int b = blockIdx.x * (blockDim.x / PI_HEAD_DIM) + threadIdx.x / PI_HEAD_DIM;
+    const int d = threadIdx.x % PI_HEAD_DIM;
+    const int ctx = max(ctx_len[seq], 0);
+    const int n_blocks = min((ctx + B - 1) / B, max_blocks);
+    if (b >= n_blocks) return;
+    const int valid = min(B, ctx - b * B);
+    const __nv_bfloat16* k = kv + seq * seq_stride_elems +
+                             (static_cast<long long>(b) * Hkv + h_star) * 2ll * B * PI_HEAD_DIM + d;
+    __nv_bfloat16 lo = k[0], hi = k[0];
+    for (int t = 1; t < valid; ++t) {
+        const __nv_bfloat16 x = k[static_cast<size_t>(t) * PI_HEAD_DIM];
+        if (__bfloat162float(x) < __bfloat162float(lo)) lo = x;
+        if (__bfloat162float(x) > __bfloat162float(hi)) hi = x;
+    }
+    __nv_bfloat16* out = digest + (static_cast<size_t>(seq) * max_blocks + b) * 2 * PI_HEAD_DIM + d;
+    out[0] = lo;
+    out[PI_HEAD_DIM] = hi;
+}
+
+__global__ void table_init_kernel(const int32_t* resident, int32_t* table, int32_t* slot_block, uint32_t* slot_stamp,
+                                  int C, int max_blocks) {
+    const int seq = blockIdx.x;
+    int32_t* t = table + static_cast<size_t>(seq) * max_blocks;
+    for (int i = threadIdx.x; i < max_blocks; i += blockDim.x) t[i] = -1;
+    __syncthreads();
+    for (int s = threadIdx.x; s < C; s += blockDim.x) {
+        int b = resident[static_cast<size_t>(seq) * C + s];
+        if (b >= max_blocks) b = -1;
+        slot_block[static_cast<size_t>(seq) * C + s] = b < 0 ? -1 : b;
+        slot_stamp[static_cast<size_t>(seq) * C + s] = 0u;
+        if (b >= 0) t[b] = s;
+    }
+}
+
+}  // namespace
+
+int pi_launch_build_digests(pi_ctx* c, int h_star, int batch, const void* kv, int64_t stride,
+                            const int32_t* ctx_len, void* digest, cudaStream_t stream) {
+    const int threads = 256, per_cta = threads / PI_HEAD_DIM;
+    dim3 grid((c->cfg.max_blocks + per_cta - 1) / per_cta, batch);
+    build_digests_kernel<<<grid, threads, 0, stream>>>(static_cast<const __nv_bfloat16*>(kv), stride / 2, ctx_len,
+                                                       static_cast<__nv_bfloat16*>(digest), h_star,
+                                                       c->cfg.n_kv_heads, c->cfg.block_tokens, c->cfg.max_blocks);
+    PI_CUDA_TRY(cudaGetLastError());
+    return PI_OK;
+}
+
+int pi_launch_table_init(pi_ctx* c, int batch, const int32_t* resident, int32_t* table, int32_t* slot_block,
+                         uint32_t* slot_stamp, cudaStream_t stream) {
+    table_init_kernel<<<batch, 256, 0, stream>>>(resident, table, slot_block, slot_stamp, c->cfg.pool_slots,
+                                                 c->cfg.max_blocks);
+    PI_CUDA_TRY(cudaGetLastError());
+    return PI_OK;
+}
