@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Benchmark of the decode recall path (score -> select -> diff -> recall -> attention).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c2] [--impl reference]
+
+One "step" is one decode step of the whole batch: every layer runs one layer-step of the
+path.  The metric is layer-steps per second.  Rank 0 prints ONE JSON line.
+
+  value        inputs (queries) already in HBM, the pipelined two-stream form
+  e2e          the same through DecodeSession with the queries coming from pinned host memory
+               and the outputs copied back to pinned host memory inside the timed region
+  roofline     the kernel that dominates the step (the recall pull, bound by the host link)
+  rooflines    the HBM-bound kernels (attention, scoring) against the measured HBM copy rate
+  cpu_baseline the CPU oracle timed on a bounded sample of the same workload
+
+With --gpus N > 1 every rank runs its own batch of sequences (weak scaling, no collective
+on the data path); the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+import numpy as np
+import torch
+
+METRIC = "decode layer-steps/s (select+recall+attn); recall GB/s vs measured H2D peak"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks() -> dict:
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return dict(hbm_gbs=float(d["hbm_gbs"]), source="measured")
+    return dict(hbm_gbs=FALLBACK_HBM_GBS, source="fallback")
+
+
+def mem_available_bytes() -> int:
+    for line in Path("/proc/meminfo").read_text().splitlines():
+        if line.startswith("MemAvailable"):
+            return int(line.split()[1]) * 1024
+    return 0
+
+
+class ClockSampler:
+    """nvidia-smi sampling of SM clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+def build_session(cfg, rank: int, host_layers_arg: int, world: int):
+    from paper_2609_34555_b200 import PulseInfer
+    from paper_2609_34555_b200.runner import DecodeSession
+    from workloads import generate as gen
+
+    per_layer = cfg.batch * cfg.n_blocks * cfg.block_bytes
+    if host_layers_arg > 0:
+        R = min(host_layers_arg, cfg.n_layers)
+    else:
+        budget = 0.55 * mem_available_bytes() / max(1, world)
+        R = int(max(1, min(cfg.n_layers, budget // per_layer)))
+    pi = PulseInfer.from_workload(cfg)
+    sess = DecodeSession(pi, cfg.batch, cfg.n_layers, host_layers=R)
+    sess.ctx_len.fill_(cfg.ctx)
+    dev = sess.device
+    for l in range(cfg.n_layers):
+        kv = gen.make_kv(cfg, l, device=dev) if l < R else None
+        res = torch.from_numpy(gen.initial_resident(cfg, l)).to(dev)
+        sess.load_layer(l, kv, res)
+        del kv
+    torch.cuda.synchronize()
+    return pi, sess, R
+
+
+def make_all_queries(cfg, steps: int, device) -> torch.Tensor:
+    """[steps][n_layers][batch][Hq][D] bf16 on `device`."""
+    from workloads import generate as gen
+    per_layer = [gen.make_queries(cfg, l, steps, device=device) for l in range(cfg.n_layers)]
+    return torch.stack(per_layer, dim=1).contiguous()
+
+
+def run_ours(args) -> dict:
+    from paper_2609_34555_b200 import h2d_copy_ms
+    from paper_2609_34555_b200.runner import StageTimer
+    from workloads import get_config
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    base = get_config(args.config)
+    cfg = base.replace(seed=base.seed + 7919 * rank)
+    if args.layers > 0:                       # profiling only: fewer layers of the same shape
+        cfg = cfg.replace(n_layers=min(args.layers, cfg.n_layers), name=f"{cfg.name}[{args.layers} layers only]")
+    K, W = args.steps, max(3, args.warmup)
+
+    t_setup = time.time()
+    pi, sess, R = build_session(cfg, rank, args.host_layers, world)
+    n_e2e = K if not args.no_e2e else 0
+    n_serial = min(K, 4)
+    q_all = make_all_queries(cfg, W + K + n_serial + n_e2e, dev)
+    setup_s = time.time() - t_setup
+
+    # pinned host -> device copy peak, measured in this run (1 GiB, best of 10)
+    probe_bytes = min(1 << 30, sess.host_kv[0].numel() * 2)
+    probe_src = sess.host_kv[0].view(-1)[: probe_bytes // 2]
+    probe_dst = torch.empty(probe_bytes // 2, dtype=torch.bfloat16, device=dev)
+    h2d_gbs = probe_bytes / (h2d_copy_ms(probe_src, probe_dst, reps=10) * 1e-3) / 1e9
+    del probe_dst
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    t = 0
+    for _ in range(W):
+        sess.decode_step(q_all[t]); t += 1
+    barrier()
+    pi.stats(reset=True)
+
+    # ---------------- timed region: K pipelined decode steps, inputs resident in HBM
+    sampler = ClockSampler(local)
+    sampler.start()
+    timer = StageTimer()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(K):
+        sess.decode_step(q_all[t], timer=timer); t += 1
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        import torch.distributed as dist
+        tm = torch.tensor([ms], device=dev)
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+        ms = float(tm.item())
+    stats = pi.stats(reset=True)
+    stages = timer.summary()
+    status = pi.status()
+    if status[0] != 0:
+        raise RuntimeError(f"device status after the timed region: {status}")
+
+    # ---------------- serial form (one stream), a few steps, for the per-stage picture
+    ser_timer = StageTimer()
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0.record()
+    for _ in range(n_serial):
+        sess.decode_step(q_all[t], overlapped=False, timer=ser_timer); t += 1
+    s1.record()
+    torch.cuda.synchronize()
+    serial_ms = s0.elapsed_time(s1) / max(1, n_serial)
+    ser_stats = pi.stats(reset=True)
+    ser = ser_timer.summary()
+
+    # ---------------- end to end: queries from pinned host memory, outputs back to it
+    e2e = None
+    if n_e2e:
+        q_host = q_all[t:t + n_e2e].cpu().pin_memory()
+        out_host = torch.empty(sess.out.shape, dtype=torch.bfloat16, pin_memory=True)
+        q_dev = torch.empty_like(q_all[0])
+        barrier()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for i in range(n_e2e):
+            sess.decode_step_from_host(q_host[i], out_host, q_dev)
+        a1.record()
+        barrier()
+        e2e_ms = a0.elapsed_time(a1)
+        if world > 1:
+            import torch.distributed as dist
+            tm = torch.tensor([e2e_ms], device=dev)
+            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+            e2e_ms = float(tm.item())
+        e2e = dict(value=world * n_e2e * cfg.n_layers / (e2e_ms * 1e-3), unit="layer-steps/s",
+                   h2d_bytes_per_step=int(q_dev.numel() * 2), d2h_bytes_per_step=int(out_host.numel() * 2),
+                   note="host KV store is read by the recall kernel in both forms")
+        pi.stats(reset=True)
+
+    peaks = measured_peaks()
+    n_launch = K * cfg.n_layers
+    recall_bytes = stats["missing_blocks"] * cfg.block_bytes
+    recall_s = stages["recall"]["total_ms"] * 1e-3
+    attn_bytes_launch = stats["selected_blocks"] / max(1, n_launch) * cfg.block_bytes + 2 * cfg.batch * cfg.n_q_heads * 128 * 2
+    score_bytes_launch = cfg.batch * cfg.n_blocks * 512 + cfg.batch * cfg.group * 128 * 2
+    def hbm_entry(name, bytes_launch, st, traffic):
+        ach = bytes_launch / (st["mean_ms"] * 1e-3) / 1e9
+        return dict(kernel=name, bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s",
+                    frac=ach / peaks["hbm_gbs"], peak_source=peaks["source"], traffic=traffic,
+                    bytes_per_launch=int(bytes_launch), mean_us=st["mean_ms"] * 1e3)
+    ser_recall_gbs = ser_stats["missing_blocks"] * cfg.block_bytes / max(1e-9, ser["recall"]["total_ms"] * 1e-3) / 1e9
+    recall_gbs = recall_bytes / max(1e-9, recall_s) / 1e9
+    line = {
+        "metric": METRIC, "value": world * K * cfg.n_layers / (ms * 1e-3), "unit": "layer-steps/s",
+        "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms / K, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: {cfg.n_layers} layers x batch {cfg.batch} x ctx {cfg.ctx}, "
+                               f"Hq/Hkv {cfg.n_q_heads}/{cfg.n_kv_heads}, block {cfg.block_tokens}, budget {cfg.budget_blocks} "
+                               f"blocks, pool {cfg.pool_slots} slots/seq/layer, AR(1) queries a={cfg.ar1}",
+                   "host_kv_layers": R, "host_kv_pinned_gb": R * cfg.batch * cfg.n_blocks * cfg.block_bytes / 2 ** 30,
+                   "l2": "inputs larger than L2 (pool reads 128 MiB and digests 16 MiB per layer-step, all layers distinct)",
+                   "pipeline": "select+diff+recall on a side stream, attention on the main stream",
+                   "sequence_layer_steps_per_s": world * K * cfg.n_layers * cfg.batch / (ms * 1e-3),
+                   "misses_per_seq_layer_step": stats["missing_blocks"] / max(1, stats["sequences"]),
+                   "setup_s": round(setup_s, 1)},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": 4 * n_launch,
+        "roofline": {"kernel": "recall_kernel", "bound": "host_link_h2d", "achieved": recall_gbs, "peak": h2d_gbs,
+                     "unit": "GB/s", "frac": recall_gbs / h2d_gbs,
+                     "peak_source": "pinned cudaMemcpyAsync H2D of 1 GiB, best of 10, this run (nominal 64 GB/s PCIe Gen5 x16)",
+                     "traffic": None, "bytes_per_launch": int(recall_bytes / max(1, n_launch)),
+                     "mean_us": stages["recall"]["mean_ms"] * 1e3,
+                     "alone": {"achieved": ser_recall_gbs, "frac": ser_recall_gbs / h2d_gbs}},
+        "rooflines": [hbm_entry("attn_kernel", attn_bytes_launch, stages["attn"], None),
+                      hbm_entry("score_select_kernel", score_bytes_launch, stages["score_select"], None),
+                      dict(hbm_entry("attn_kernel (serial form, nothing else running)", attn_bytes_launch, ser["attn"], None)),
+                      dict(hbm_entry("score_select_kernel (serial form)", score_bytes_launch, ser["score_select"], None))],
+        "stages_us": {k: v["mean_ms"] * 1e3 for k, v in stages.items()},
+        "serial": {"layer_steps_per_s": cfg.n_layers / (serial_ms * 1e-3),
+                   "stages_us": {k: v["mean_ms"] * 1e3 for k, v in ser.items()}},
+        "h2d_peak_gbs": h2d_gbs,
+    }
+    if rank == 0 and not args.no_cpu and world == 1:
+        line["cpu_baseline"] = cpu_baseline(cfg, sess, budget_s=args.cpu_seconds)
+    return line if rank == 0 else {}
+
+
+def oracle_state(cfg, sess, layers):
+    """numpy state of the oracle for some layers, initialised like the GPU's was."""
+    import oracle
+    from workloads import generate as gen
+    st = {}
+    for l in layers:
+        host = sess.host_region(l)
+        kvb = oracle.bits(host)                              # view of the pinned store
+        h = cfg.solo_head(l)
+        dg = np.stack([oracle.build_digest(kvb[s], cfg.ctx, h) for s in range(cfg.batch)])
+        res = gen.initial_resident(cfg, l)
+        table = np.full((cfg.batch, cfg.n_blocks), -1, np.int32)
+        pool = np.zeros((cfg.batch, cfg.pool_slots) + kvb.shape[2:], np.uint16)
+        for s in range(cfg.batch):
+            ok = res[s] >= 0
+            table[s, res[s][ok]] = np.nonzero(ok)[0]
+            pool[s, ok] = kvb[s, res[s][ok]]
+        st[l] = dict(kvb=kvb, digest=dg, table=table, slot_block=res.copy(),
+                     slot_stamp=np.zeros((cfg.batch, cfg.pool_slots), np.uint32), pool=pool, h=h)
+    return st
+
+
+def cpu_baseline(cfg, sess, budget_s: float) -> dict:
+    """The oracle, as it stands, on a bounded sample: whole-batch layer-steps of the first
+    layers with the same queries, until about `budget_s` seconds of CPU work are done."""
+    import oracle
+    from workloads import generate as gen
+    layers = list(range(min(2, cfg.n_layers)))
+    st = oracle_state(cfg, sess, layers)
+    q = {l: oracle.bits(gen.make_queries(cfg, l, 64, device="cpu")) for l in layers}
+    ctx_len = np.full(cfg.batch, cfg.ctx, np.int32)
+    done, t0, step = 0, time.perf_counter(), 0
+    while True:
+        step += 1
+        for l in layers:
+            s = st[l]
+            r = oracle.layer_step(ctx_len, cfg.n_blocks, cfg.block_tokens, cfg.n_kv_heads, s["h"], cfg.budget_blocks,
+                                  cfg.n_sink_blocks, cfg.n_local_blocks, step, q[l][(step - 1) % 64], s["digest"],
+                                  s["kvb"], s["table"], s["slot_block"], s["slot_stamp"], s["pool"])
+            assert r["rc"] == 0
+            done += 1
+        el = time.perf_counter() - t0
+        if el >= budget_s or step >= 64:
+            break
+    return dict(value=done / el, unit="layer-steps/s", cores=oracle.num_threads(), kind="oracle",
+                sample=f"{done} whole-batch layer-steps (layers {layers}, {step} decode steps) in {el:.1f} s; "
+                       f"host: {os.cpu_count()} cores")
+
+
+def run_reference(args) -> dict:
+    """The reference arm: the CPU oracle timed on bounded samples of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return {}
+    import oracle
+    from workloads import generate as gen, get_config
+    cfg = get_config(args.config)
+    K, W = args.steps, max(3, args.warmup)
+    # a bounded sample: one layer of the model, the whole batch, one layer-step per bench step
+    layer = 0
+    kv = gen.make_kv(cfg, layer)
+    kvb = oracle.bits(kv)
+    h = cfg.solo_head(layer)
+    dg = np.stack([oracle.build_digest(kvb[s], cfg.ctx, h) for s in range(cfg.batch)])
+    res = gen.initial_resident(cfg, layer)
+    table = np.full((cfg.batch, cfg.n_blocks), -1, np.int32)
+    pool = np.zeros((cfg.batch, cfg.pool_slots) + kvb.shape[2:], np.uint16)
+    for s in range(cfg.batch):
+        ok = res[s] >= 0
+        table[s, res[s][ok]] = np.nonzero(ok)[0]
+        pool[s, ok] = kvb[s, res[s][ok]]
+    sb, stmp = res.copy(), np.zeros((cfg.batch, cfg.pool_slots), np.uint32)
+    q = oracle.bits(gen.make_queries(cfg, layer, W + K))
+    ctx_len = np.full(cfg.batch, cfg.ctx, np.int32)
+    per = max(1, min(cfg.n_layers, args.ref_layer_steps))
+
+    def one(step):
+        for _ in range(per):
+            r = oracle.layer_step(ctx_len, cfg.n_blocks, cfg.block_tokens, cfg.n_kv_heads, h, cfg.budget_blocks,
+                                  cfg.n_sink_blocks, cfg.n_local_blocks, step, q[step - 1], dg, kvb, table, sb, stmp, pool)
+            assert r["rc"] == 0
+    for t in range(W):
+        one(t + 1)
+    t0 = time.perf_counter()
+    for t in range(W, W + K):
+        one(t + 1)
+    el = time.perf_counter() - t0
+    value = K * per / el
+    sample = (f"each step = {per} whole-batch layer-step(s) of layer 0 (of {cfg.n_layers} per decode step); "
+              f"host: {os.cpu_count()} cores")
+    return {"impl": "reference", "metric": METRIC, "value": value, "unit": "layer-steps/s", "n_gpus": 1,
+            "steps": K, "warmup": W, "ms_per_step": el / K * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: CPU oracle, {sample}"},
+            "cpu_baseline": dict(value=value, unit="layer-steps/s", cores=oracle.num_threads(), kind="oracle", sample=sample),
+            "e2e": {"value": value, "unit": "layer-steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="c2")
+    ap.add_argument("--host-layers", type=int, default=0, help="distinct host KV regions (0 = as many as fit)")
+    ap.add_argument("--layers", type=int, default=0, help="cut the layer stack (for profiler captures only)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--ref-layer-steps", type=int, default=1)
+    args = ap.parse_args()
+    line = run_reference(args) if args.impl == "reference" else run_ours(args)
+    if line:
+        print(json.dumps(line), flush=True)
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1 and args.impl != "reference":
+        import torch.distributed as dist
+        if dist.is_initialized():
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -155,6 +155,10 @@ int pi_h2d_copy_ms(const void* host_pinned, void* dev, int64_t bytes, int reps, 
  * or list, position, offending value.  Reads a pinned mirror: call after the stream
  * has been synchronised.  pi_clear_status resets it. */
 int pi_get_status(pi_ctx* ctx, int32_t out[8]);
+/* Counters accumulated by pi_diff_misses since creation or the last reset: out[0] = sequences
+ * diffed, out[1] = selected blocks, out[2] = missing blocks (= blocks recalled), out[3] = extents
+ * emitted.  Synchronises the device. */
+int pi_get_stats(pi_ctx* ctx, int64_t out[4], int reset);
 int pi_clear_status(pi_ctx* ctx);
 const char* pi_strerror(int code);
 

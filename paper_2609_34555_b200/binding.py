@@ -24,7 +24,7 @@ EXTENT_DTYPE = torch.int32      # a pi_extent is four int32: src_unit, dst_unit,
 
 EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_diff_misses", "pi_recall_gather_scatter",
            "pi_sparse_decode_attn", "pi_build_digests", "pi_table_init", "pi_h2d_copy_ms",
-           "pi_get_status", "pi_clear_status", "pi_strerror"]
+           "pi_get_status", "pi_get_stats", "pi_clear_status", "pi_strerror"]
 
 
 class PiConfig(ctypes.Structure):
@@ -63,6 +63,7 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.pi_table_init.argtypes = [c_void_p, c_int, i32p, i32p, i32p, u32p, vp]
     lib.pi_h2d_copy_ms.argtypes = [vp, vp, c_int64, c_int, POINTER(c_float)]
     lib.pi_get_status.argtypes = [c_void_p, POINTER(c_int32 * 8)]
+    lib.pi_get_stats.argtypes = [c_void_p, POINTER(c_int64 * 4), c_int]
     lib.pi_clear_status.argtypes = [c_void_p]
     lib.pi_strerror.argtypes = [c_int]
     lib.pi_strerror.restype = c_char_p
@@ -206,6 +207,11 @@ class PulseInfer:
         out = (c_int32 * 8)()
         _check("pi_get_status", self._lib.pi_get_status(self._ctx, ctypes.byref(out)))
         return list(out)
+
+    def stats(self, reset: bool = False) -> dict:
+        out = (c_int64 * 4)()
+        _check("pi_get_stats", self._lib.pi_get_stats(self._ctx, ctypes.byref(out), int(reset)))
+        return dict(sequences=out[0], selected_blocks=out[1], missing_blocks=out[2], extents=out[3])
 
     def clear_status(self) -> None:
         _check("pi_clear_status", self._lib.pi_clear_status(self._ctx))

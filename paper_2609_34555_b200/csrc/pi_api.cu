@@ -68,6 +68,7 @@ extern "C" int pi_create(const pi_config* cfg, pi_ctx** out) {
               cudaMalloc(&c->attn_part_o, n_part * cfg->n_q_heads * PI_HEAD_DIM * sizeof(float)) == cudaSuccess &&
               cudaMalloc(&c->attn_part_ml, n_part * cfg->n_q_heads * 2 * sizeof(float)) == cudaSuccess &&
               cudaMalloc(&c->status_flag_dev, sizeof(int)) == cudaSuccess &&
+              cudaMalloc(&c->stats_dev, 4 * sizeof(unsigned long long)) == cudaSuccess &&
               cudaHostAlloc(&host, 8 * sizeof(int32_t), cudaHostAllocMapped) == cudaSuccess;
     if (ok) {
         c->status_host = static_cast<volatile int32_t*>(host);
@@ -77,6 +78,7 @@ extern "C" int pi_create(const pi_config* cfg, pi_ctx** out) {
              cudaMemset(c->sel_counters, 0, nb * sizeof(unsigned int)) == cudaSuccess &&
              cudaMemset(c->attn_counters, 0, nb * sizeof(unsigned int)) == cudaSuccess &&
              cudaMemset(c->status_flag_dev, 0, sizeof(int)) == cudaSuccess &&
+             cudaMemset(c->stats_dev, 0, 4 * sizeof(unsigned long long)) == cudaSuccess &&
              cudaDeviceSynchronize() == cudaSuccess;
         c->status_host_devptr = static_cast<int32_t*>(alias);
     }
@@ -98,6 +100,7 @@ extern "C" int pi_destroy(pi_ctx* c) {
     cudaFree(c->attn_part_o);
     cudaFree(c->attn_part_ml);
     cudaFree(c->status_flag_dev);
+    cudaFree(c->stats_dev);
     if (c->status_host) cudaFreeHost(const_cast<int32_t*>(c->status_host));
     (void)cudaGetLastError();
     std::free(c->solo_head);
@@ -238,6 +241,16 @@ extern "C" int pi_h2d_copy_ms(const void* host_pinned, void* dev, int64_t bytes,
 extern "C" int pi_get_status(pi_ctx* ctx, int32_t out[8]) {
     if (!ctx || !out) return PI_ERR_INVALID_ARG;
     for (int i = 0; i < 8; ++i) out[i] = ctx->status_host[i];
+    return PI_OK;
+}
+
+extern "C" int pi_get_stats(pi_ctx* ctx, int64_t out[4], int reset) {
+    if (!ctx || !out) return PI_ERR_INVALID_ARG;
+    unsigned long long h[4];
+    PI_CUDA_TRY(cudaDeviceSynchronize());
+    PI_CUDA_TRY(cudaMemcpy(h, ctx->stats_dev, sizeof(h), cudaMemcpyDeviceToHost));
+    if (reset) PI_CUDA_TRY(cudaMemset(ctx->stats_dev, 0, sizeof(h)));
+    for (int i = 0; i < 4; ++i) out[i] = static_cast<int64_t>(h[i]);
     return PI_OK;
 }
 

@@ -26,6 +26,7 @@ struct DiffParams {
     pi_extent* list;
     int32_t* count;
     pi_status_ref st;
+    unsigned long long* stats;
     uint32_t step;
     int B, K, C, Cpad, n_sink, n_local, max_blocks;
 };
@@ -194,7 +195,13 @@ diff_kernel(DiffParams p) {
             }
         }
     }
-    if (tid == 0) p.count[seq] = n_ext;
+    if (tid == 0) {
+        p.count[seq] = n_ext;
+        atomicAdd(p.stats + 0, 1ull);
+        atomicAdd(p.stats + 1, static_cast<unsigned long long>(cnt));
+        atomicAdd(p.stats + 2, static_cast<unsigned long long>(too_small ? 0 : n_miss));
+        atomicAdd(p.stats + 3, static_cast<unsigned long long>(n_ext));
+    }
 }
 
 }  // namespace
@@ -207,6 +214,7 @@ int pi_launch_diff(pi_ctx* c, int batch, uint32_t step, const int32_t* ctx_len, 
     p.table = table; p.slot_block = slot_block; p.slot_stamp = slot_stamp;
     p.sel_slots = sel_slots; p.list = list; p.count = count;
     p.st = pi_status_of(c);
+    p.stats = c->stats_dev;
     p.step = step;
     p.B = c->cfg.block_tokens; p.K = c->cfg.budget_blocks; p.C = c->cfg.pool_slots;
     int cpad = 2;

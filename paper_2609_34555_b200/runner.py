@@ -91,3 +91,124 @@ class RecallPath:
         ev.record(self.side)
         main.wait_event(ev)
         self.attention(layer, buf, q, ctx_len, out, lse)
+
+
+class StageTimer:
+    """CUDA events around each call of a decode step, on the stream the call runs on."""
+
+    STAGES = ("score_select", "diff", "recall", "attn")
+
+    def __init__(self):
+        self.pairs = {s: [] for s in self.STAGES}
+
+    def mark(self, stream) -> torch.cuda.Event:
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record(stream)
+        return ev
+
+    def add(self, stage: str, a: torch.cuda.Event, b: torch.cuda.Event) -> None:
+        self.pairs[stage].append((a, b))
+
+    def summary(self) -> dict:
+        """Per stage: launches, mean and total milliseconds (call after a synchronize)."""
+        out = {}
+        for s, lst in self.pairs.items():
+            ms = [a.elapsed_time(b) for a, b in lst]
+            out[s] = dict(launches=len(ms), total_ms=float(sum(ms)), mean_ms=float(sum(ms) / max(1, len(ms))))
+        return out
+
+
+class DecodeSession:
+    """All layers of one batch of offloaded sequences: per-layer device buffers, the pinned
+    host store, and the pipelined decode step (selection + diff + recall of every layer on a
+    side stream, attention on the main stream as soon as that layer's recall has landed).
+
+    `host_layers` < n_layers lets several layers share one region of the host store (layer l
+    reads region l % host_layers) when host memory is short; digests, tables and pools stay
+    per layer."""
+
+    def __init__(self, pi: PulseInfer, batch: int, n_layers: int, host_layers: Optional[int] = None,
+                 device="cuda", keep_scores: bool = False):
+        c = pi.cfg
+        self.pi, self.batch, self.n_layers = pi, batch, n_layers
+        self.host_layers = n_layers if host_layers is None else max(1, min(host_layers, n_layers))
+        self.device = torch.device(device)
+        self.bufs = [LayerBuffers(pi, batch, device, keep_scores) for _ in range(n_layers)]
+        shape = (batch, c.max_blocks, c.n_kv_heads, 2, c.block_tokens, c.head_dim)
+        self.host_kv = [torch.empty(shape, dtype=torch.bfloat16, pin_memory=True) for _ in range(self.host_layers)]
+        self.out = torch.zeros((n_layers, batch, c.n_q_heads, c.head_dim), dtype=torch.bfloat16, device=device)
+        self.ctx_len = torch.zeros((batch,), dtype=torch.int32, device=device)
+        self.main = torch.cuda.current_stream(self.device)
+        self.side = torch.cuda.Stream(self.device)
+        self._ev_recall = [torch.cuda.Event() for _ in range(n_layers)]
+        self._ev_attn = [torch.cuda.Event() for _ in range(n_layers)]
+        self._ev_start = torch.cuda.Event()
+        self._path = RecallPath(pi)
+        self.step_count = 0
+
+    def host_region(self, layer: int) -> torch.Tensor:
+        return self.host_kv[layer % self.host_layers]
+
+    def load_layer(self, layer: int, kv_dev: Optional[torch.Tensor], resident: torch.Tensor) -> None:
+        """kv_dev (device copy of the layer's keys/values) is stored into the host region when
+        given; digests are built from it, tables from `resident`, and the resident blocks are
+        pulled back from the host store into the pool."""
+        host = self.host_region(layer)
+        if kv_dev is not None:
+            host.copy_(kv_dev, non_blocking=False)
+        self._path.prepare_layer(layer, self.bufs[layer], host, self.ctx_len, resident,
+                                 kv_for_digest=kv_dev)
+
+    def decode_step(self, q: torch.Tensor, overlapped: bool = True, timer: Optional[StageTimer] = None) -> torch.Tensor:
+        """q: device bf16 [n_layers][batch][Hq][D].  Returns self.out ([n_layers][batch][Hq][D]);
+        valid once the main stream has caught up."""
+        pi = self.pi
+        self.step_count += 1
+        step = self.step_count
+        main = torch.cuda.current_stream(self.device)
+        side = self.side if overlapped else main
+        if overlapped:
+            self._ev_start.record(main)
+            side.wait_event(self._ev_start)
+        for l in range(self.n_layers):
+            b, host = self.bufs[l], self.host_region(l)
+            if overlapped and step > 1:
+                side.wait_event(self._ev_attn[l])          # last step's attention still reads this layer's pool
+            t0 = timer.mark(side) if timer else None
+            pi.score_select(l, q[l], b.digest, self.ctx_len, b.sel_blocks, b.sel_count, b.scores, stream=side)
+            t1 = timer.mark(side) if timer else None
+            pi.diff_misses(l, step, self.ctx_len, b.sel_blocks, b.sel_count, b.block_table, b.slot_block,
+                           b.slot_stamp, b.sel_slots, b.recall_list, b.recall_count, stream=side)
+            t2 = timer.mark(side) if timer else None
+            pi.recall_gather_scatter(l, host, b.pool, b.recall_list, b.recall_count, stream=side)
+            t3 = timer.mark(side) if timer else None
+            if overlapped:
+                self._ev_recall[l].record(side)
+                main.wait_event(self._ev_recall[l])
+            t4 = timer.mark(main) if timer else None
+            pi.sparse_decode_attn(l, q[l], b.pool, b.sel_slots, b.sel_blocks, b.sel_count, self.ctx_len,
+                                  self.out[l], None, stream=main)
+            t5 = timer.mark(main) if timer else None
+            if overlapped:
+                self._ev_attn[l].record(main)
+            if timer:
+                timer.add("score_select", t0, t1); timer.add("diff", t1, t2)
+                timer.add("recall", t2, t3); timer.add("attn", t4, t5)
+        return self.out
+
+    def decode_step_from_host(self, q_host: torch.Tensor, out_host: torch.Tensor, q_dev: torch.Tensor) -> None:
+        """End-to-end form: queries come from pinned host memory, results go back to pinned
+        host memory; both copies are enqueued on the main stream around the step."""
+        q_dev.copy_(q_host, non_blocking=True)
+        self.decode_step(q_dev, overlapped=True)
+        out_host.copy_(self.out, non_blocking=True)
+
+    def miss_blocks(self) -> int:
+        """Units recalled by the last step (synchronises; bookkeeping for reports)."""
+        total = 0
+        for b in self.bufs:
+            cnt = b.recall_count
+            lst = b.recall_list
+            idx = torch.arange(lst.shape[1], device=lst.device)[None, :] < cnt[:, None]
+            total += int((lst[:, :, 2] * idx).sum().item())
+        return total
