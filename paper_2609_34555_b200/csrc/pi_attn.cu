@@ -113,6 +113,83 @@ __device__ __forceinline__ int seq_of_unit(const int* pref, int batch, int u) {
     return lo;
 }
 
+// Merge of the split-K partials of one sequence by warp h for its G query heads.  Lane i
+// fetches (m, l) of segment i, the warp agrees on the maximum, and the weighted sum of the
+// partial outputs runs over segments with eight independent 16-byte loads in flight per lane
+// (4 heads x 2 segments); each lane owns 4 of the 128 channels.
+__device__ __forceinline__ void merge_partials(const AttnParams& p, int seq, int h, int c_first, int c_last, int lane) {
+    const int n_seg = c_last - c_first + 1;
+    const size_t slot0 = static_cast<size_t>(c_first) + seq;
+    for (int g0 = 0; g0 < p.G; g0 += 4) {
+        float M[4], L[4];
+        float4 acc[4];
+#pragma unroll
+        for (int gi = 0; gi < 4; ++gi) { M[gi] = -INFINITY; L[gi] = 0.f; acc[gi] = make_float4(0.f, 0.f, 0.f, 0.f); }
+        const size_t head0 = static_cast<size_t>(h) * p.G + g0;
+        for (int s0 = 0; s0 < n_seg; s0 += 32) {
+            const int sg = s0 + lane;
+#pragma unroll
+            for (int gi = 0; gi < 4; ++gi)
+                if (sg < n_seg && g0 + gi < p.G)
+                    M[gi] = fmaxf(M[gi], __ldcg(p.part_ml + ((slot0 + sg) * p.Hq + head0 + gi) * 2));
+        }
+#pragma unroll
+        for (int gi = 0; gi < 4; ++gi)
+#pragma unroll
+            for (int o = 16; o; o >>= 1) M[gi] = fmaxf(M[gi], __shfl_xor_sync(0xffffffffu, M[gi], o));
+        for (int s0 = 0; s0 < n_seg; s0 += 32) {
+            const int sg = s0 + lane;
+            float w[4];
+#pragma unroll
+            for (int gi = 0; gi < 4; ++gi) {
+                w[gi] = 0.f;
+                if (sg < n_seg && g0 + gi < p.G) {
+                    const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((slot0 + sg) * p.Hq + head0 + gi) * 2));
+                    w[gi] = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M[gi]);
+                    L[gi] += w[gi] * ml.y;
+                }
+            }
+            const int cnt = min(32, n_seg - s0);
+            for (int k = 0; k < cnt; k += 2) {
+                float4 v[2][4];
+#pragma unroll
+                for (int kk = 0; kk < 2; ++kk)
+#pragma unroll
+                    for (int gi = 0; gi < 4; ++gi) {
+                        v[kk][gi] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (k + kk < cnt && g0 + gi < p.G)
+                            v[kk][gi] = __ldcg(reinterpret_cast<const float4*>(
+                                            p.part_o + ((slot0 + s0 + k + kk) * p.Hq + head0 + gi) * PI_HEAD_DIM) + lane);
+                    }
+#pragma unroll
+                for (int kk = 0; kk < 2; ++kk)
+#pragma unroll
+                    for (int gi = 0; gi < 4; ++gi) {
+                        const float wk = __shfl_sync(0xffffffffu, w[gi], (k + kk) & 31);
+                        acc[gi].x += wk * v[kk][gi].x; acc[gi].y += wk * v[kk][gi].y;
+                        acc[gi].z += wk * v[kk][gi].z; acc[gi].w += wk * v[kk][gi].w;
+                    }
+            }
+        }
+#pragma unroll
+        for (int gi = 0; gi < 4; ++gi) {
+#pragma unroll
+            for (int o = 16; o; o >>= 1) L[gi] += __shfl_xor_sync(0xffffffffu, L[gi], o);
+            if (g0 + gi >= p.G) continue;
+            const float inv = L[gi] > 0.f ? 1.f / L[gi] : 0.f;
+            const size_t gh = static_cast<size_t>(seq) * p.Hq + head0 + gi;
+            __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc[gi].x * inv, acc[gi].y * inv);
+            __nv_bfloat162 hi2 = __floats2bfloat162_rn(acc[gi].z * inv, acc[gi].w * inv);
+            uint2 pk;
+            pk.x = *reinterpret_cast<uint32_t*>(&lo2);
+            pk.y = *reinterpret_cast<uint32_t*>(&hi2);
+            *reinterpret_cast<uint2*>(p.out + gh * PI_HEAD_DIM + lane * 4) = pk;
+            if (p.lse && lane == 0)
+                p.lse[gh] = L[gi] > 0.f ? (M[gi] + log2f(L[gi])) * 0.6931471805599453f : -INFINITY;
+        }
+    }
+}
+
 template <int NT>
 __global__ void __launch_bounds__(288, 1)
 attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
@@ -387,33 +464,7 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
                 seg_round += 2;
                 if (*s_last) {
                     __threadfence();
-                    // merge: warp h reduces its G heads over the n_seg partials; lane owns 4 channels
-                    for (int g = 0; g < p.G; ++g) {
-                        const size_t head = static_cast<size_t>(h) * p.G + g;
-                        float M = -INFINITY;
-                        for (int cc = c_first; cc <= c_last; ++cc)
-                            M = fmaxf(M, __ldcg(p.part_ml + ((static_cast<size_t>(cc) + seq) * p.Hq + head) * 2));
-                        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                        float L = 0.f;
-                        for (int cc = c_first; cc <= c_last; ++cc) {
-                            const size_t gh = (static_cast<size_t>(cc) + seq) * p.Hq + head;
-                            const float mi_ = __ldcg(p.part_ml + gh * 2), li_ = __ldcg(p.part_ml + gh * 2 + 1);
-                            const float w = (mi_ == -INFINITY) ? 0.f : exp2f(mi_ - M);
-                            const float4 v = __ldcg(reinterpret_cast<const float4*>(p.part_o + gh * PI_HEAD_DIM) + lane);
-                            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
-                            L += w * li_;
-                        }
-                        const float inv = L > 0.f ? 1.f / L : 0.f;
-                        const size_t go = (static_cast<size_t>(seq) * p.Hq + head) * PI_HEAD_DIM + lane * 4;
-                        __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-                        __nv_bfloat162 hi2 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-                        uint2 pk;
-                        pk.x = *reinterpret_cast<uint32_t*>(&lo2);
-                        pk.y = *reinterpret_cast<uint32_t*>(&hi2);
-                        *reinterpret_cast<uint2*>(p.out + go) = pk;
-                        if (p.lse && lane == 0)
-                            p.lse[static_cast<size_t>(seq) * p.Hq + head] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
-                    }
+                    merge_partials(p, seq, h, c_first, c_last, lane);
                 }
                 // the flag is rewritten only after every warp passed the next pair of barriers
             }

@@ -124,20 +124,26 @@ diff_kernel(DiffParams p) {
     const bool too_small = s_ncand < n_miss;
 
     if (n_miss > 0 && !too_small) {
-        // 3. bitonic sort of the candidate keys (ascending)
+        // 3. bitonic sort of the candidate keys (ascending).  Warp w owns elements
+        // [32*E*w, 32*E*(w+1)), so exchanges at distance < 32*E stay inside one warp and need
+        // only a warp barrier; the few longer ones are fenced by CTA barriers.
+        const int E = max(1, p.Cpad / DIFF_THREADS), wspan = 32 * E;
+        const int lane = tid & 31, warp = tid >> 5;
         for (int k = 2; k <= p.Cpad; k <<= 1) {
             for (int j = k >> 1; j > 0; j >>= 1) {
-                for (int i = tid; i < p.Cpad; i += DIFF_THREADS) {
-                    const int l = i ^ j;
-                    if (l > i) {
+                if (j >= wspan) __syncthreads();
+                for (int e = 0; e < E; ++e) {
+                    const int i = (warp * E + e) * 32 + lane, l = i ^ j;
+                    if (l > i && l < p.Cpad) {
                         const unsigned long long a = keys[i], b = keys[l];
                         const bool up = (i & k) == 0;
                         if ((a > b) == up) { keys[i] = b; keys[l] = a; }
                     }
                 }
-                __syncthreads();
+                if (j >= wspan) __syncthreads(); else __syncwarp();
             }
         }
+        __syncthreads();
         // 4. i-th miss takes the i-th candidate
         for (int i = tid; i < n_miss; i += DIFF_THREADS) {
             const int j = s_miss[i];

@@ -19,12 +19,13 @@
 
 namespace {
 
-constexpr int SCORE_THREADS = 256;
+constexpr int SCORE_THREADS = 512;
 constexpr int SCORE_WARPS = SCORE_THREADS / 32;
-constexpr int SCORE_CHUNK = 128;                 // blocks per CTA
-constexpr int BLOCKS_PER_ITER = 8;               // per warp: 8 independent 16-byte loads per lane
+constexpr int BLOCKS_PER_WARP = 8;               // 8 independent 16-byte loads per lane
+constexpr int SCORE_CHUNK = SCORE_WARPS * BLOCKS_PER_WARP;   // 128 blocks (64 KB of digests) per CTA
 constexpr int BINS = PI_SELECT_BINS;
 constexpr int BINS_PER_THREAD = BINS / SCORE_THREADS;
+constexpr int RESOLVE_MAX = 32;                  // bucket sizes one warp resolves by direct ranking
 
 struct SelParams {
     const __nv_bfloat16* q;
@@ -37,6 +38,11 @@ struct SelParams {
     pi_status_ref st;
     int h_star, Hq, G, B, K, n_sink, n_local, max_blocks;
 };
+
+// Shared arrays that one thread walks with a stride of several words are stored with one
+// pad word every 32 entries, which keeps both the strided and the unit-stride walks free
+// of bank conflicts.
+__device__ __forceinline__ int padded(int i) { return i + (i >> 5); }
 
 __device__ __forceinline__ uint32_t float_key(float s) {
     uint32_t u = __float_as_uint(s + 0.0f);       // -0 -> +0
@@ -62,7 +68,7 @@ __device__ __forceinline__ float dot8(uint4 v, const float (&w)[8]) {
     return s0 + s1;
 }
 
-// Block-wide exclusive scan helpers (SCORE_THREADS threads, all must call).
+// Block-wide exclusive scan (SCORE_THREADS threads, all must call).
 __device__ __forceinline__ unsigned block_excl_scan(unsigned v, unsigned* warp_tot, unsigned& total) {
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     unsigned inc = v;
@@ -74,29 +80,72 @@ __device__ __forceinline__ unsigned block_excl_scan(unsigned v, unsigned* warp_t
     __syncthreads();                               // warp_tot may still be read from a previous call
     if (lane == 31) warp_tot[w] = inc;
     __syncthreads();
-    unsigned base = 0, tot = 0;
+    unsigned mine = lane < SCORE_WARPS ? warp_tot[lane] : 0u;
+    unsigned pre = mine;
 #pragma unroll
-    for (int i = 0; i < SCORE_WARPS; ++i) {
-        unsigned t = warp_tot[i];
-        if (i < w) base += t;
-        tot += t;
+    for (int o = 1; o < SCORE_WARPS; o <<= 1) {
+        unsigned t = __shfl_up_sync(0xffffffffu, pre, o);
+        if (lane >= o) pre += t;
     }
-    total = tot;
+    total = __shfl_sync(0xffffffffu, pre, SCORE_WARPS - 1);
+    const unsigned base = w == 0 ? 0u : __shfl_sync(0xffffffffu, pre, w - 1);
     return base + inc - v;
 }
 
-__global__ void __launch_bounds__(SCORE_THREADS)
+__global__ void __launch_bounds__(SCORE_THREADS, 2)
 score_select_kernel(SelParams p) {
-    extern __shared__ uint32_t keys[];             // [n_blocks] in the selecting CTA
-    __shared__ unsigned hist[BINS];
+    extern __shared__ uint32_t keys[];             // [padded(n_blocks)] in the selecting CTA
+    __shared__ unsigned hist[BINS + BINS / 32 + 1];
     __shared__ unsigned warp_tot[SCORE_WARPS];
     __shared__ uint32_t red_lo[SCORE_WARPS], red_hi[SCORE_WARPS];
+    __shared__ uint32_t cand_key[RESOLVE_MAX];
+    __shared__ int cand_idx[RESOLVE_MAX];
     __shared__ uint32_t sh_lo, sh_hi;
-    __shared__ unsigned sh_need, sh_cnt;
+    __shared__ unsigned sh_need, sh_cnt, sh_ncand;
     __shared__ int sh_last;
 
     const int seq = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    // ---------------- phase 1: scores of this CTA's chunk.  Every load (digest rows, the
+    // group's queries, the context length) is issued before anything waits: digest rows up
+    // to max_blocks are allocated, so they are read unguarded and masked at the store.
+    const int b0 = blockIdx.x * SCORE_CHUNK + warp * BLOCKS_PER_WARP;
+    const uint4* dg = p.digest + static_cast<size_t>(seq) * p.max_blocks * 32;   // 32 uint4 per block
+    uint4 v[BLOCKS_PER_WARP];
+#pragma unroll
+    for (int i = 0; i < BLOCKS_PER_WARP; ++i) {
+        v[i] = make_uint4(0, 0, 0, 0);
+        if (b0 + i < p.max_blocks) v[i] = ld_stream16(dg + static_cast<size_t>(b0 + i) * 32 + lane);
+    }
+    // lanes 0-15 hold Q- for channels 8*lane.., lanes 16-31 hold Q+ for channels 8*(lane-16)..
+    float w[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) w[i] = 0.f;
+    {
+        const int d0 = (lane & 15) * 8;
+        const bool plus = lane >= 16;
+        const __nv_bfloat16* qh = p.q + (static_cast<size_t>(seq) * p.Hq + static_cast<size_t>(p.h_star) * p.G) * PI_HEAD_DIM + d0;
+        // the group's query rows are fetched four at a time so their latencies overlap
+        for (int g0 = 0; g0 < p.G; g0 += 4) {
+            uint4 qv[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                qv[j] = make_uint4(0, 0, 0, 0);
+                if (g0 + j < p.G) qv[j] = *reinterpret_cast<const uint4*>(qh + static_cast<size_t>(g0 + j) * PI_HEAD_DIM);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&qv[j]);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float2 f = __bfloat1622float2(h2[i]);
+                    w[2 * i] += plus ? fmaxf(f.x, 0.f) : fminf(f.x, 0.f);
+                    w[2 * i + 1] += plus ? fmaxf(f.y, 0.f) : fminf(f.y, 0.f);
+                }
+            }
+        }
+    }
     int ctx = p.ctx_len[seq];
     if (ctx < 0) ctx = 0;
     int n_blocks = (ctx + p.B - 1) / p.B;
@@ -104,78 +153,49 @@ score_select_kernel(SelParams p) {
         if (tid == 0 && blockIdx.x == 0) pi_report(p.st, PI_ERR_CAPACITY, PI_STAGE_SELECT, seq, n_blocks, p.max_blocks);
         n_blocks = p.max_blocks;
     }
-
-    // ---------------- phase 1: scores of this CTA's chunk
-    const int c0 = blockIdx.x * SCORE_CHUNK;
-    if (c0 < n_blocks) {
-        // lanes 0-15 hold Q- for channels 8*lane.., lanes 16-31 hold Q+ for channels 8*(lane-16)..
-        float w[8];
+    {
+        float s[BLOCKS_PER_WARP];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) w[i] = 0.f;
-        const int d0 = (lane & 15) * 8;
-        const bool plus = lane >= 16;
-        const __nv_bfloat16* qh = p.q + (static_cast<size_t>(seq) * p.Hq + static_cast<size_t>(p.h_star) * p.G) * PI_HEAD_DIM + d0;
-        for (int g = 0; g < p.G; ++g) {
-            uint4 v = *reinterpret_cast<const uint4*>(qh + static_cast<size_t>(g) * PI_HEAD_DIM);
-            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&v);
+        for (int i = 0; i < BLOCKS_PER_WARP; ++i) s[i] = dot8(v[i], w);
+        // transposed warp reduction: 8 values x 32 lanes -> lane group (lane>>2) owns block (lane>>2)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                float2 f = __bfloat1622float2(h2[i]);
-                w[2 * i] += plus ? fmaxf(f.x, 0.f) : fminf(f.x, 0.f);
-                w[2 * i + 1] += plus ? fmaxf(f.y, 0.f) : fminf(f.y, 0.f);
-            }
+        for (int i = 0; i < 4; ++i) {
+            const bool up = lane & 16;
+            float send = up ? s[i] : s[i + 4];
+            float keep = up ? s[i + 4] : s[i];
+            s[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
         }
-        const uint4* dg = p.digest + static_cast<size_t>(seq) * p.max_blocks * 32;   // 32 uint4 per block
-        for (int b0 = c0 + warp * BLOCKS_PER_ITER; b0 < c0 + SCORE_CHUNK && b0 < n_blocks;
-             b0 += SCORE_WARPS * BLOCKS_PER_ITER) {
-            uint4 v[BLOCKS_PER_ITER];
 #pragma unroll
-            for (int i = 0; i < BLOCKS_PER_ITER; ++i) {
-                v[i] = make_uint4(0, 0, 0, 0);
-                if (b0 + i < n_blocks) v[i] = ld_stream16(dg + static_cast<size_t>(b0 + i) * 32 + lane);
-            }
-            float s[BLOCKS_PER_ITER];
-#pragma unroll
-            for (int i = 0; i < BLOCKS_PER_ITER; ++i) s[i] = dot8(v[i], w);
-            // transposed warp reduction: 8 values x 32 lanes -> lane group (lane>>2) owns block (lane>>2)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const bool up = lane & 16;
-                float send = up ? s[i] : s[i + 4];
-                float keep = up ? s[i + 4] : s[i];
-                s[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
-            }
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                const bool up = lane & 8;
-                float send = up ? s[i] : s[i + 2];
-                float keep = up ? s[i + 2] : s[i];
-                s[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
-            }
-            {
-                const bool up = lane & 4;
-                float send = up ? s[0] : s[1];
-                float keep = up ? s[1] : s[0];
-                s[0] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-            }
-            s[0] += __shfl_xor_sync(0xffffffffu, s[0], 2);
-            s[0] += __shfl_xor_sync(0xffffffffu, s[0], 1);
-            const int b = b0 + (lane >> 2);
-            if ((lane & 3) == 0 && b < n_blocks) p.scores[static_cast<size_t>(seq) * p.max_blocks + b] = s[0];
+        for (int i = 0; i < 2; ++i) {
+            const bool up = lane & 8;
+            float send = up ? s[i] : s[i + 2];
+            float keep = up ? s[i + 2] : s[i];
+            s[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
         }
+        {
+            const bool up = lane & 4;
+            float send = up ? s[0] : s[1];
+            float keep = up ? s[1] : s[0];
+            s[0] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+        }
+        s[0] += __shfl_xor_sync(0xffffffffu, s[0], 2);
+        s[0] += __shfl_xor_sync(0xffffffffu, s[0], 1);
+        const int b = b0 + (lane >> 2);
+        if ((lane & 3) == 0 && b < n_blocks) p.scores[static_cast<size_t>(seq) * p.max_blocks + b] = s[0];
     }
 
     // ---------------- ticket: the last CTA of the sequence selects
-    __threadfence();
+    // (the CTA barrier orders every thread's score stores before thread 0's fence and ticket)
     __syncthreads();
     if (tid == 0) {
+        __threadfence();
         unsigned t = atomicAdd(&p.counters[seq], 1u);
         sh_last = (t == gridDim.x - 1);
         if (sh_last) p.counters[seq] = 0;           // ready for the next launch
+        __threadfence();
     }
     __syncthreads();
     if (!sh_last) return;
-    __threadfence();
 
     // ---------------- phase 2: selection
     const int m_lo = min(p.n_sink, n_blocks);
@@ -188,7 +208,7 @@ score_select_kernel(SelParams p) {
     const float* sc = p.scores + static_cast<size_t>(seq) * p.max_blocks;
     for (int i = tid; i < n_blocks; i += SCORE_THREADS) {
         uint32_t key = float_key(__ldcg(sc + i));
-        keys[i] = key;
+        keys[padded(i)] = key;
         if (i >= m_lo && i < m_hi) { kmin = min(kmin, key); kmax = max(kmax, key); }
     }
 #pragma unroll
@@ -198,16 +218,16 @@ score_select_kernel(SelParams p) {
     }
     if (lane == 0) { red_lo[warp] = kmin; red_hi[warp] = kmax; }
     __syncthreads();
-    if (tid == 0) {
+    {
         uint32_t a = red_lo[0], b = red_hi[0];
+#pragma unroll
         for (int i = 1; i < SCORE_WARPS; ++i) { a = min(a, red_lo[i]); b = max(b, red_hi[i]); }
-        sh_lo = a; sh_hi = b; sh_need = k; sh_cnt = static_cast<unsigned>(n_mid);
+        kmin = a; kmax = b;
     }
-    __syncthreads();
 
     // Narrow [lo, hi] until keys > hi are all winners and the first `need` keys (by index)
     // inside [lo, hi] complete the set.
-    uint32_t lo = sh_lo, hi = sh_hi;
+    uint32_t lo = kmin, hi = kmax;
     unsigned need = k;
     if (k > 0 && k < static_cast<unsigned>(n_mid)) {
         for (int pass = 0; pass < 4; ++pass) {
@@ -215,44 +235,74 @@ score_select_kernel(SelParams p) {
             if (range == 0) break;                   // every key left is equal: ties by index
             const int bits = 32 - __clz(range);
             const int shift = bits > 11 ? bits - 11 : 0;
-            for (int i = tid; i < BINS; i += SCORE_THREADS) hist[i] = 0;
+            for (int i = tid; i < BINS + BINS / 32 + 1; i += SCORE_THREADS) hist[i] = 0;
             __syncthreads();
             for (int i = m_lo + tid; i < m_hi; i += SCORE_THREADS) {
-                const uint32_t key = keys[i];
-                if (key >= lo && key <= hi) atomicAdd(&hist[(key - lo) >> shift], 1u);
+                const uint32_t key = keys[padded(i)];
+                if (key >= lo && key <= hi) atomicAdd(&hist[padded((key - lo) >> shift)], 1u);
             }
             __syncthreads();
-            // suffix sums from the top bin: thread t owns bins [t*BPT, t*BPT+BPT), reversed order
-            const int top = BINS - 1 - tid * BINS_PER_THREAD;          // my highest bin
-            unsigned local = 0;
+            // suffix sums from the top bin: thread t owns bins [top - BPT + 1, top], top = BINS-1 - t*BPT
+            const int top = BINS - 1 - tid * BINS_PER_THREAD;
+            unsigned hb[BINS_PER_THREAD], local = 0;
 #pragma unroll
-            for (int j = 0; j < BINS_PER_THREAD; ++j) local += hist[top - j];
+            for (int j = 0; j < BINS_PER_THREAD; ++j) { hb[j] = hist[padded(top - j)]; local += hb[j]; }
             unsigned total;
             const unsigned above = block_excl_scan(local, warp_tot, total);  // keys in bins above mine
             if (above < need && need <= above + local) {
                 unsigned acc = above;
+#pragma unroll
                 for (int j = 0; j < BINS_PER_THREAD; ++j) {
-                    const unsigned h = hist[top - j];
-                    if (need <= acc + h) {
+                    if (need > acc && need <= acc + hb[j]) {
                         const uint32_t nlo = lo + (static_cast<uint32_t>(top - j) << shift);
                         const uint32_t span = shift ? ((1u << shift) - 1u) : 0u;
                         sh_lo = nlo;
                         sh_hi = (hi - nlo < span) ? hi : nlo + span;
                         sh_need = need - acc;
-                        sh_cnt = h;
-                        break;
+                        sh_cnt = hb[j];
                     }
-                    acc += h;
+                    acc += hb[j];
                 }
+                sh_ncand = 0;
             }
             __syncthreads();
             lo = sh_lo; hi = sh_hi; need = sh_need;
             const unsigned cnt = sh_cnt;
             if (shift == 0 || cnt == need) break;
+            if (cnt <= RESOLVE_MAX) {
+                // few keys left in the bucket: one warp ranks them by (key descending, index ascending)
+                for (int i = m_lo + tid; i < m_hi; i += SCORE_THREADS) {
+                    const uint32_t key = keys[padded(i)];
+                    if (key >= lo && key <= hi) {
+                        const unsigned pos = atomicAdd(&sh_ncand, 1u);
+                        cand_key[pos] = key;
+                        cand_idx[pos] = i;
+                    }
+                }
+                __syncthreads();
+                if (warp == 0) {
+                    const bool have = lane < static_cast<int>(cnt);
+                    const uint32_t mk = have ? cand_key[lane] : 0u;
+                    const int mi = have ? cand_idx[lane] : 0x7fffffff;
+                    unsigned rank = 0;
+                    for (unsigned j = 0; j < cnt; ++j) {
+                        const uint32_t ok = cand_key[j];
+                        const int oi = cand_idx[j];
+                        rank += (ok > mk || (ok == mk && oi < mi)) ? 1u : 0u;
+                    }
+                    // the need-th best candidate fixes the threshold key; ties at it go by index
+                    const unsigned is_tau = __ballot_sync(0xffffffffu, have && rank == need - 1);
+                    const uint32_t tau = __shfl_sync(0xffffffffu, mk, __ffs(is_tau) - 1);
+                    const unsigned eq_taken = __popc(__ballot_sync(0xffffffffu, have && mk == tau && rank < need));
+                    if (lane == 0) { sh_lo = tau; sh_hi = tau; sh_need = eq_taken; }
+                }
+                __syncthreads();
+                lo = sh_lo; hi = sh_hi; need = sh_need;
+                break;
+            }
         }
     } else if (k == 0) {
-        lo = 0xffffffffu; hi = 0xffffffffu; need = 0;       // nothing from the middle (keys are never all-ones for finite scores)
-        // keys equal to 0xffffffff cannot occur for finite scores; `need` = 0 excludes them anyway
+        lo = 0xffffffffu; hi = 0xffffffffu; need = 0;       // nothing from the middle
     } else {
         need = static_cast<unsigned>(n_mid);                // everything: [lo, hi] already spans all keys
     }
@@ -263,7 +313,7 @@ score_select_kernel(SelParams p) {
     unsigned c_sure = 0, c_eq = 0;
     for (int i = i0; i < i1; ++i) {
         if (i < m_lo || i >= m_hi) { ++c_sure; continue; }
-        const uint32_t key = keys[i];
+        const uint32_t key = keys[padded(i)];
         if (k > 0 && key > hi) ++c_sure;
         else if (k > 0 && key >= lo) ++c_eq;
     }
@@ -276,7 +326,7 @@ score_select_kernel(SelParams p) {
         unsigned pos = sure_b + min(eq_b, need);
         if (i < m_lo || i >= m_hi) { take = true; ++sure_b; }
         else {
-            const uint32_t key = keys[i];
+            const uint32_t key = keys[padded(i)];
             if (k > 0 && key > hi) { take = true; ++sure_b; }
             else if (k > 0 && key >= lo) { take = eq_b < need; ++eq_b; }
             else take = false;
@@ -310,7 +360,7 @@ int pi_launch_score_select(pi_ctx* c, int h_star, int batch, const void* q, cons
     p.n_sink = c->cfg.n_sink_blocks;
     p.n_local = c->cfg.n_local_blocks;
     p.max_blocks = c->cfg.max_blocks;
-    const size_t smem = static_cast<size_t>(c->cfg.max_blocks) * sizeof(uint32_t);
+    const size_t smem = (static_cast<size_t>(c->cfg.max_blocks) + c->cfg.max_blocks / 32 + 1) * sizeof(uint32_t);
     if (smem > 40 * 1024)
         PI_CUDA_TRY(cudaFuncSetAttribute(score_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
     dim3 grid((c->cfg.max_blocks + SCORE_CHUNK - 1) / SCORE_CHUNK, batch);

@@ -98,8 +98,12 @@ class StageTimer:
 
     STAGES = ("score_select", "diff", "recall", "attn")
 
-    def __init__(self):
-        self.pairs = {s: [] for s in self.STAGES}
+    def __init__(self, stages=None):
+        self.stages = tuple(stages) if stages else self.STAGES
+        self.pairs = {s: [] for s in self.stages}
+
+    def wants(self, stage: str) -> bool:
+        return stage in self.pairs
 
     def mark(self, stream) -> torch.cuda.Event:
         ev = torch.cuda.Event(enable_timing=True)
@@ -120,8 +124,9 @@ class StageTimer:
 
 class DecodeSession:
     """All layers of one batch of offloaded sequences: per-layer device buffers, the pinned
-    host store, and the pipelined decode step (selection + diff + recall of every layer on a
-    side stream, attention on the main stream as soon as that layer's recall has landed).
+    host store, and the pipelined decode step (selection + diff of every layer on one side
+    stream, the recall pulls on a second, attention on the main stream as soon as that layer's
+    recall has landed).
 
     `host_layers` < n_layers lets several layers share one region of the host store (layer l
     reads region l % host_layers) when host memory is short; digests, tables and pools stay
@@ -140,6 +145,8 @@ class DecodeSession:
         self.ctx_len = torch.zeros((batch,), dtype=torch.int32, device=device)
         self.main = torch.cuda.current_stream(self.device)
         self.side = torch.cuda.Stream(self.device)
+        self.side2 = torch.cuda.Stream(self.device)
+        self._ev_diff = [torch.cuda.Event() for _ in range(n_layers)]
         self._ev_recall = [torch.cuda.Event() for _ in range(n_layers)]
         self._ev_attn = [torch.cuda.Event() for _ in range(n_layers)]
         self._ev_start = torch.cuda.Event()
@@ -161,39 +168,51 @@ class DecodeSession:
 
     def decode_step(self, q: torch.Tensor, overlapped: bool = True, timer: Optional[StageTimer] = None) -> torch.Tensor:
         """q: device bf16 [n_layers][batch][Hq][D].  Returns self.out ([n_layers][batch][Hq][D]);
-        valid once the main stream has caught up."""
+        valid once the current stream has caught up.
+
+        Overlapped form: three streams.  Selection and diff of every layer run ahead on one
+        stream, the recall pulls follow on a second one (the host link stays busy back to
+        back), and each layer's attention runs on the current stream once its recall landed."""
         pi = self.pi
         self.step_count += 1
         step = self.step_count
         main = torch.cuda.current_stream(self.device)
-        side = self.side if overlapped else main
+        sel_s = self.side if overlapped else main
+        rec_s = self.side2 if overlapped else main
         if overlapped:
             self._ev_start.record(main)
-            side.wait_event(self._ev_start)
+            sel_s.wait_event(self._ev_start)
         for l in range(self.n_layers):
             b, host = self.bufs[l], self.host_region(l)
             if overlapped and step > 1:
-                side.wait_event(self._ev_attn[l])          # last step's attention still reads this layer's pool
-            t0 = timer.mark(side) if timer else None
-            pi.score_select(l, q[l], b.digest, self.ctx_len, b.sel_blocks, b.sel_count, b.scores, stream=side)
-            t1 = timer.mark(side) if timer else None
+                sel_s.wait_event(self._ev_attn[l])         # last step's attention still reads this layer's lists and pool
+            tm = timer
+            t0 = tm.mark(sel_s) if tm and tm.wants("score_select") else None
+            pi.score_select(l, q[l], b.digest, self.ctx_len, b.sel_blocks, b.sel_count, b.scores, stream=sel_s)
+            t1 = tm.mark(sel_s) if tm and (tm.wants("score_select") or tm.wants("diff")) else None
             pi.diff_misses(l, step, self.ctx_len, b.sel_blocks, b.sel_count, b.block_table, b.slot_block,
-                           b.slot_stamp, b.sel_slots, b.recall_list, b.recall_count, stream=side)
-            t2 = timer.mark(side) if timer else None
-            pi.recall_gather_scatter(l, host, b.pool, b.recall_list, b.recall_count, stream=side)
-            t3 = timer.mark(side) if timer else None
+                           b.slot_stamp, b.sel_slots, b.recall_list, b.recall_count, stream=sel_s)
+            t2 = tm.mark(sel_s) if tm and tm.wants("diff") else None
             if overlapped:
-                self._ev_recall[l].record(side)
+                self._ev_diff[l].record(sel_s)
+                rec_s.wait_event(self._ev_diff[l])
+            t2r = tm.mark(rec_s) if tm and tm.wants("recall") else None
+            pi.recall_gather_scatter(l, host, b.pool, b.recall_list, b.recall_count, stream=rec_s)
+            t3 = tm.mark(rec_s) if tm and tm.wants("recall") else None
+            if overlapped:
+                self._ev_recall[l].record(rec_s)
                 main.wait_event(self._ev_recall[l])
-            t4 = timer.mark(main) if timer else None
+            t4 = tm.mark(main) if tm and tm.wants("attn") else None
             pi.sparse_decode_attn(l, q[l], b.pool, b.sel_slots, b.sel_blocks, b.sel_count, self.ctx_len,
                                   self.out[l], None, stream=main)
-            t5 = timer.mark(main) if timer else None
+            t5 = tm.mark(main) if tm and tm.wants("attn") else None
             if overlapped:
                 self._ev_attn[l].record(main)
-            if timer:
-                timer.add("score_select", t0, t1); timer.add("diff", t1, t2)
-                timer.add("recall", t2, t3); timer.add("attn", t4, t5)
+            if tm:
+                if t0 is not None: tm.add("score_select", t0, t1)
+                if t2 is not None: tm.add("diff", t1, t2)
+                if t2r is not None: tm.add("recall", t2r, t3)
+                if t4 is not None: tm.add("attn", t4, t5)
         return self.out
 
     def decode_step_from_host(self, q_host: torch.Tensor, out_host: torch.Tensor, q_dev: torch.Tensor) -> None:
