@@ -44,6 +44,7 @@ extern "C" {
 #define PI_ERR_TIMEOUT         (-7)   /* a bounded device-side wait ran out          */
 #define PI_ERR_INDEX_RANGE     (-8)   /* a block / slot index read from a list is out of range */
 #define PI_ERR_CAPACITY        (-9)   /* a count read from device memory exceeds its capacity  */
+#define PI_ERR_STATIC_LIMIT   (-10)  /* batch or block count beyond the fixed scratch of pi_score_select_noalloc */
 
 typedef struct pi_ctx pi_ctx;
 
@@ -88,6 +89,33 @@ int pi_destroy(pi_ctx* ctx);
 int pi_score_select(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* digest_dev,
                     const int32_t* ctx_len_dev, int32_t* sel_blocks_dev, int32_t* sel_count_dev,
                     float* scores_dev, void* stream);
+
+/* pi_score_select for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; this exists for the library's users.)  Some code runs where cudaMalloc is off
+ * limits: a plug-in inside a serving engine that hands out all device memory itself, a callback
+ * on a latency-critical path where an allocation could stall or fail, a process whose memory
+ * pool is already fully committed.  Such a caller cannot call pi_create, which allocates the
+ * score buffer and the per-sequence tickets.  This entry point needs no context: it computes the
+ * same selection as pi_score_select (same kernel, same results bit for bit) and keeps that
+ * scratch in a fixed array inside the library image instead.
+ *   Limits: batch <= 64 and max_blocks <= 8192, else PI_ERR_STATIC_LIMIT and nothing runs.  The
+ *   array takes 2 MiB + 512 B on every GPU that loads the library, until the process exits.
+ *   The call allocates nothing and frees nothing (no cudaMalloc / cudaFree, no library routine
+ *   that allocates); it enqueues two small memsets and the kernel on `stream` and returns.
+ *   The first call on each device also looks up the array's device address, with that device
+ *   current; make that first call outside any stream capture.
+ *   All calls on a device share the one array, and it keeps the previous call's contents; the
+ *   words that must start at zero are cleared on `stream` before the kernel.  Two calls whose
+ *   kernels can overlap on the GPU (different streams, no dependency) race on it: order them.
+ *   Model shape and budget come as plain arguments (meaning as in pi_config); solo_head is the
+ *   retrieval KV head of this layer.  q, digest, ctx_len, sel_blocks, sel_count: as pi_score_select.
+ *   status_dev: NULL, or device int32[8] that receives what pi_get_status would report for this
+ *   call ([0] code, [1] stage, [2..4] coordinates; [7] is used internally); cleared on `stream`. */
+int pi_score_select_noalloc(int batch, int n_q_heads, int n_kv_heads, int block_tokens,
+                            int budget_blocks, int n_sink_blocks, int n_local_blocks, int max_blocks,
+                            int solo_head, const void* q_dev, const void* digest_dev,
+                            const int32_t* ctx_len_dev, int32_t* sel_blocks_dev, int32_t* sel_count_dev,
+                            int32_t* status_dev, void* stream);
 
 /* Step 2 of the workflow (Sec. 2.2): B_recall = B_topk \ B_gpu against the
  * device-resident block table, victim choice (least recently selected slot, ties to

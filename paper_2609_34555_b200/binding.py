@@ -18,11 +18,11 @@ OK = 0
 ERR_NAMES = {
     -1: "PI_ERR_INVALID_ARG", -2: "PI_ERR_BAD_ALIGN", -3: "PI_ERR_UNSUPPORTED_DIM",
     -4: "PI_ERR_POOL_TOO_SMALL", -5: "PI_ERR_NOT_PINNED", -6: "PI_ERR_CUDA", -7: "PI_ERR_TIMEOUT",
-    -8: "PI_ERR_INDEX_RANGE", -9: "PI_ERR_CAPACITY",
+    -8: "PI_ERR_INDEX_RANGE", -9: "PI_ERR_CAPACITY", -10: "PI_ERR_STATIC_LIMIT",
 }
 EXTENT_DTYPE = torch.int32      # a pi_extent is four int32: src_unit, dst_unit, n_units, units_before
 
-EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_diff_misses", "pi_recall_gather_scatter",
+EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_score_select_noalloc", "pi_diff_misses", "pi_recall_gather_scatter",
            "pi_sparse_decode_attn", "pi_build_digests", "pi_table_init", "pi_h2d_copy_ms",
            "pi_get_status", "pi_get_stats", "pi_clear_status", "pi_strerror"]
 
@@ -56,6 +56,7 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.pi_create.argtypes = [POINTER(PiConfig), POINTER(c_void_p)]
     lib.pi_destroy.argtypes = [c_void_p]
     lib.pi_score_select.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, vp, vp]
+    lib.pi_score_select_noalloc.argtypes = [c_int] * 9 + [vp, vp, i32p, i32p, i32p, i32p, vp]
     lib.pi_diff_misses.argtypes = [c_void_p, c_int, c_int, c_uint32, i32p, i32p, i32p, i32p, i32p, u32p, i32p, vp, i32p, vp]
     lib.pi_recall_gather_scatter.argtypes = [c_void_p, c_int, c_int, c_int, vp, c_int64, vp, c_int64, vp, c_int32, i32p, c_int64, vp]
     lib.pi_sparse_decode_attn.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, i32p, vp, vp, vp]
@@ -104,6 +105,23 @@ def h2d_copy_ms(host_pinned: torch.Tensor, dev: torch.Tensor, reps: int = 10) ->
     ms = c_float(0)
     _check("pi_h2d_copy_ms", load_library().pi_h2d_copy_ms(host_pinned.data_ptr(), dev.data_ptr(), nbytes, reps, ctypes.byref(ms)))
     return float(ms.value)
+
+
+def score_select_noalloc(q, digest, ctx_len, sel_blocks, sel_count, *, n_kv_heads: int, block_tokens: int,
+                         budget_blocks: int, n_sink_blocks: int, n_local_blocks: int, solo_head: int,
+                         status=None, stream=None) -> None:
+    """Selection without a context and without any device allocation, for callers that are not
+    allowed to allocate (an engine that owns all device memory, a callback on a hot path).
+    Same results as PulseInfer.score_select.  batch <= 64 and max_blocks <= 8192; calls on one
+    device share a fixed scratch array inside the library, so do not let two of them overlap."""
+    batch, n_q_heads = q.shape[0], q.shape[1]
+    max_blocks = digest.shape[1]
+    _check("pi_score_select_noalloc", load_library().pi_score_select_noalloc(
+        batch, n_q_heads, n_kv_heads, block_tokens, budget_blocks, n_sink_blocks, n_local_blocks, max_blocks,
+        solo_head, _dev(q, torch.bfloat16, "q"), _dev(digest, torch.bfloat16, "digest"),
+        _dev(ctx_len, torch.int32, "ctx_len"), _dev(sel_blocks, torch.int32, "sel_blocks"),
+        _dev(sel_count, torch.int32, "sel_count"),
+        None if status is None else _dev(status, torch.int32, "status"), _stream(stream)))
 
 
 class PulseInfer:

@@ -275,6 +275,7 @@ extern "C" const char* pi_strerror(int code) {
         case PI_ERR_TIMEOUT: return "bounded device wait ran out";
         case PI_ERR_INDEX_RANGE: return "index read from a device list is out of range";
         case PI_ERR_CAPACITY: return "count read from device memory exceeds capacity";
+        case PI_ERR_STATIC_LIMIT: return "batch or max_blocks exceeds the fixed scratch of pi_score_select_noalloc (64 x 8192)";
         default: return "unknown error";
     }
 }

@@ -368,3 +368,88 @@ int pi_launch_score_select(pi_ctx* c, int h_star, int batch, const void* q, cons
     PI_CUDA_TRY(cudaGetLastError());
     return PI_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// Allocation-free variant of the call above, for callers that must not allocate device
+// memory (see the declaration in pulseinfer.h).  The scores and the per-sequence tickets,
+// which the regular call keeps in memory that pi_create allocated, live in this fixed
+// array instead.  Every GPU that loads the library holds one copy (2 MiB + 512 B) until the
+// process exits.  The array's name is only a host-side handle: the device address comes from
+// cudaGetSymbolAddress, once per device, on that device's first call.
+#include <mutex>
+
+constexpr int PI_NOALLOC_MAX_BATCH = 64;
+constexpr int PI_NOALLOC_MAX_BLOCKS = 8192;
+constexpr size_t PI_NOALLOC_HEAD_BYTES = 512;      // [0,256) status words, [256,512) tickets
+constexpr size_t PI_NOALLOC_BYTES =
+    PI_NOALLOC_HEAD_BYTES + static_cast<size_t>(PI_NOALLOC_MAX_BATCH) * PI_NOALLOC_MAX_BLOCKS * sizeof(float);
+static __device__ __align__(256) unsigned char pi_noalloc_scratch[PI_NOALLOC_BYTES];
+
+namespace {
+constexpr int NOALLOC_MAX_DEVICES = 64;
+std::mutex g_noalloc_mu;
+unsigned char* g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {};
+}  // namespace
+
+extern "C" int pi_score_select_noalloc(int batch, int n_q_heads, int n_kv_heads, int block_tokens,
+                                       int budget_blocks, int n_sink_blocks, int n_local_blocks,
+                                       int max_blocks, int solo_head, const void* q_dev,
+                                       const void* digest_dev, const int32_t* ctx_len_dev,
+                                       int32_t* sel_blocks_dev, int32_t* sel_count_dev,
+                                       int32_t* status_dev, void* stream) {
+    if (!q_dev || !digest_dev || !ctx_len_dev || !sel_blocks_dev || !sel_count_dev) return PI_ERR_INVALID_ARG;
+    if (batch < 1 || max_blocks < 1 || n_sink_blocks < 0 || n_local_blocks < 0) return PI_ERR_INVALID_ARG;
+    if (batch > PI_NOALLOC_MAX_BATCH || max_blocks > PI_NOALLOC_MAX_BLOCKS) return PI_ERR_STATIC_LIMIT;
+    if (n_kv_heads < 1 || n_q_heads < n_kv_heads || n_q_heads % n_kv_heads || n_q_heads / n_kv_heads > 16)
+        return PI_ERR_UNSUPPORTED_DIM;
+    if (block_tokens != 16 && block_tokens != 32 && block_tokens != 64) return PI_ERR_UNSUPPORTED_DIM;
+    if (budget_blocks < 1 || budget_blocks > 4096 || budget_blocks < n_sink_blocks + n_local_blocks)
+        return PI_ERR_INVALID_ARG;
+    if (solo_head < 0 || solo_head >= n_kv_heads) return PI_ERR_INVALID_ARG;
+    if (!pi_aligned16(q_dev) || !pi_aligned16(digest_dev)) return PI_ERR_BAD_ALIGN;
+
+    // set-up, once per device, with that device current: resolve the array's device address
+    int dev = -1;
+    PI_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return PI_ERR_INVALID_ARG;
+    unsigned char* base = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_noalloc_mu);
+        if (!g_noalloc_ptr[dev]) {
+            unsigned char* ptr = nullptr;
+            cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), pi_noalloc_scratch);
+            if (e != cudaSuccess || !ptr) { (void)cudaGetLastError(); return PI_ERR_CUDA; }
+            g_noalloc_ptr[dev] = ptr;
+        }
+        base = g_noalloc_ptr[dev];
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the array keeps whatever the last call left: status words and tickets must start at zero
+    PI_CUDA_TRY(cudaMemsetAsync(base, 0, PI_NOALLOC_HEAD_BYTES, s));
+    if (status_dev) PI_CUDA_TRY(cudaMemsetAsync(status_dev, 0, 8 * sizeof(int32_t), s));
+
+    SelParams p;
+    p.q = static_cast<const __nv_bfloat16*>(q_dev);
+    p.digest = static_cast<const uint4*>(digest_dev);
+    p.ctx_len = ctx_len_dev;
+    p.sel = sel_blocks_dev;
+    p.sel_count = sel_count_dev;
+    p.scores = reinterpret_cast<float*>(base + PI_NOALLOC_HEAD_BYTES);
+    p.counters = reinterpret_cast<unsigned int*>(base + 256);
+    p.st.flag = status_dev ? reinterpret_cast<int*>(status_dev + 7) : reinterpret_cast<int*>(base);
+    p.st.mirror = status_dev ? status_dev : reinterpret_cast<int32_t*>(base + 64);
+    p.h_star = solo_head;
+    p.Hq = n_q_heads;
+    p.G = n_q_heads / n_kv_heads;
+    p.B = block_tokens;
+    p.K = budget_blocks;
+    p.n_sink = n_sink_blocks;
+    p.n_local = n_local_blocks;
+    p.max_blocks = max_blocks;
+    // at most (8192 + 8192/32 + 1) keys: below the default dynamic shared-memory limit
+    const size_t smem = (static_cast<size_t>(max_blocks) + max_blocks / 32 + 1) * sizeof(uint32_t);
+    dim3 grid((max_blocks + SCORE_CHUNK - 1) / SCORE_CHUNK, batch);
+    score_select_kernel<<<grid, SCORE_THREADS, smem, s>>>(p);
+    PI_CUDA_TRY(cudaGetLastError());
+    return PI_OK;
+}
