@@ -114,25 +114,47 @@ __device__ __forceinline__ int seq_of_unit(const int* pref, int batch, int u) {
 }
 
 // Merge of the split-K partials of one sequence by warp h for its G query heads.  Lane i
-// fetches (m, l) of segment i, the warp agrees on the maximum, and the weighted sum of the
-// partial outputs runs over segments with eight independent 16-byte loads in flight per lane
-// (4 heads x 2 segments); each lane owns 4 of the 128 channels.
+// fetches (m, l) of segment i once, the warp agrees on the maximum, and the weighted sum of
+// the partial outputs runs over segments with sixteen independent 16-byte loads in flight per
+// lane (4 heads x 4 segments), the first batch issued before the weights are known; each lane
+// owns 4 of the 128 channels.
 __device__ __forceinline__ void merge_partials(const AttnParams& p, int seq, int h, int c_first, int c_last, int lane) {
     const int n_seg = c_last - c_first + 1;
     const size_t slot0 = static_cast<size_t>(c_first) + seq;
     for (int g0 = 0; g0 < p.G; g0 += 4) {
+        const size_t head0 = static_cast<size_t>(h) * p.G + g0;
         float M[4], L[4];
         float4 acc[4];
 #pragma unroll
         for (int gi = 0; gi < 4; ++gi) { M[gi] = -INFINITY; L[gi] = 0.f; acc[gi] = make_float4(0.f, 0.f, 0.f, 0.f); }
-        const size_t head0 = static_cast<size_t>(h) * p.G + g0;
+        // pass 1: maxima (one load per lane per head when n_seg <= 32)
+        float2 ml0[4];
+#pragma unroll
+        for (int gi = 0; gi < 4; ++gi) ml0[gi] = make_float2(-INFINITY, 0.f);
         for (int s0 = 0; s0 < n_seg; s0 += 32) {
             const int sg = s0 + lane;
 #pragma unroll
             for (int gi = 0; gi < 4; ++gi)
-                if (sg < n_seg && g0 + gi < p.G)
-                    M[gi] = fmaxf(M[gi], __ldcg(p.part_ml + ((slot0 + sg) * p.Hq + head0 + gi) * 2));
+                if (sg < n_seg && g0 + gi < p.G) {
+                    const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((slot0 + sg) * p.Hq + head0 + gi) * 2));
+                    if (s0 == 0) ml0[gi] = ml;
+                    M[gi] = fmaxf(M[gi], ml.x);
+                }
         }
+        // first batch of partial outputs: independent of the weights, so issued before the reduction
+        float4 v[4][4];
+        auto fetch = [&](int base_seg) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+#pragma unroll
+                for (int gi = 0; gi < 4; ++gi) {
+                    v[kk][gi] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (base_seg + kk < n_seg && g0 + gi < p.G)
+                        v[kk][gi] = __ldcg(reinterpret_cast<const float4*>(
+                                        p.part_o + ((slot0 + base_seg + kk) * p.Hq + head0 + gi) * PI_HEAD_DIM) + lane);
+                }
+        };
+        fetch(0);
 #pragma unroll
         for (int gi = 0; gi < 4; ++gi)
 #pragma unroll
@@ -144,25 +166,17 @@ __device__ __forceinline__ void merge_partials(const AttnParams& p, int seq, int
             for (int gi = 0; gi < 4; ++gi) {
                 w[gi] = 0.f;
                 if (sg < n_seg && g0 + gi < p.G) {
-                    const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((slot0 + sg) * p.Hq + head0 + gi) * 2));
+                    const float2 ml = s0 == 0 ? ml0[gi]
+                        : __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((slot0 + sg) * p.Hq + head0 + gi) * 2));
                     w[gi] = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M[gi]);
                     L[gi] += w[gi] * ml.y;
                 }
             }
             const int cnt = min(32, n_seg - s0);
-            for (int k = 0; k < cnt; k += 2) {
-                float4 v[2][4];
+            for (int k = 0; k < cnt; k += 4) {
+                if (s0 + k > 0) fetch(s0 + k);
 #pragma unroll
-                for (int kk = 0; kk < 2; ++kk)
-#pragma unroll
-                    for (int gi = 0; gi < 4; ++gi) {
-                        v[kk][gi] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (k + kk < cnt && g0 + gi < p.G)
-                            v[kk][gi] = __ldcg(reinterpret_cast<const float4*>(
-                                            p.part_o + ((slot0 + s0 + k + kk) * p.Hq + head0 + gi) * PI_HEAD_DIM) + lane);
-                    }
-#pragma unroll
-                for (int kk = 0; kk < 2; ++kk)
+                for (int kk = 0; kk < 4; ++kk)
 #pragma unroll
                     for (int gi = 0; gi < 4; ++gi) {
                         const float wk = __shfl_sync(0xffffffffu, w[gi], (k + kk) & 31);
@@ -207,6 +221,7 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + ATTN_MAX_STAGES);
     const uint32_t bar_seg = smem_u32(bars + 2 * ATTN_MAX_STAGES);
     const int SUB = p.B >> 4;
+    if (tid == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&pool_map) : "memory");
 
     // ---- unit prefix over sequences (every CTA computes the same table)
     for (int s = tid; s < p.batch; s += blockDim.x) {
@@ -302,38 +317,38 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
     // =============================== consumers: warp h owns kv head h
     const int h = warp;
     const int row = lane >> 2, colp = (lane & 3) * 2;
-    uint32_t bq[NT][8][2];
-    float o[NT][8][4], m[NT][2], l[NT][2];
     int seq = seq_of_unit(s_pref, p.batch, u0);
-    bool fresh = true;
     int seg_round = 0;
     // per-lane ldmatrix offsets inside a stage (swizzled 128-byte rows)
     const int r8 = lane & 7, mi = lane >> 3;
     const int tK = r8 + 8 * (mi & 1), cK = mi >> 1;         // K as A operand (rows = tokens)
     const int tV = r8 + 8 * (mi >> 1), cV = mi & 1;         // V^T as A operand via .trans
     const uint32_t offK = (2 * h) * 2048 + tK * 128, offV = (2 * h + 1) * 2048 + tV * 128;
+    bool alive = true;
 
-    for (int u = u0, it = 0; u < u1; ++u, ++it) {
-        while (u >= s_pref[seq + 1]) { ++seq; fresh = true; }
-        if (fresh) {
-            fresh = false;
+    // One iteration per (CTA, sequence) segment: the running softmax state lives only inside it.
+    for (int u = u0, it = 0; u < u1 && alive;) {
+        while (u >= s_pref[seq + 1]) ++seq;
+        const int seg_end = min(u1, s_pref[seq + 1]);
+        uint32_t bq[NT][8][2];
+        float o[NT][8][4], m[NT][2], l[NT][2];
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                const int g = nt * 8 + row;
-                const __nv_bfloat16* qg = p.q + (static_cast<size_t>(seq) * p.Hq + static_cast<size_t>(h) * p.G + g) * PI_HEAD_DIM + colp;
+        for (int nt = 0; nt < NT; ++nt) {
+            const int g = nt * 8 + row;
+            const __nv_bfloat16* qg = p.q + (static_cast<size_t>(seq) * p.Hq + static_cast<size_t>(h) * p.G + g) * PI_HEAD_DIM + colp;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    bq[nt][j][0] = g < p.G ? *reinterpret_cast<const uint32_t*>(qg + 16 * j) : 0u;
-                    bq[nt][j][1] = g < p.G ? *reinterpret_cast<const uint32_t*>(qg + 16 * j + 8) : 0u;
-                }
-                m[nt][0] = m[nt][1] = -INFINITY;
-                l[nt][0] = l[nt][1] = 0.f;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) o[nt][i][0] = o[nt][i][1] = o[nt][i][2] = o[nt][i][3] = 0.f;
+            for (int j = 0; j < 8; ++j) {
+                bq[nt][j][0] = g < p.G ? *reinterpret_cast<const uint32_t*>(qg + 16 * j) : 0u;
+                bq[nt][j][1] = g < p.G ? *reinterpret_cast<const uint32_t*>(qg + 16 * j + 8) : 0u;
             }
+            m[nt][0] = m[nt][1] = -INFINITY;
+            l[nt][0] = l[nt][1] = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) o[nt][i][0] = o[nt][i][1] = o[nt][i][2] = o[nt][i][3] = 0.f;
         }
+      for (; u < seg_end; ++u, ++it) {
         const int st = it % p.stages;
-        if (!mbar_wait(bar_full + 8 * st, (it / p.stages) & 1, s_abort)) break;
+        if (!mbar_wait(bar_full + 8 * st, (it / p.stages) & 1, s_abort)) { alive = false; break; }
         const int nvalid = s_nvalid[st];
         const uint32_t base = ring + st * stage_bytes;
 
@@ -400,9 +415,11 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_empty + 8 * st);
+      }
+        if (!alive) break;
 
-        // ---- end of this CTA's segment of the sequence?
-        if (u + 1 == u1 || u + 1 == s_pref[seq + 1]) {
+        // ---- end of this CTA's segment of the sequence
+        {
             const int c_first = cta_of_unit(s_pref[seq], U, P), c_last = cta_of_unit(s_pref[seq + 1] - 1, U, P);
             const int n_seg = c_last - c_first + 1;
 #pragma unroll
@@ -448,22 +465,23 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
                         }
                         if (row == 0) { p.part_ml[gh * 2] = m[nt][e]; p.part_ml[gh * 2 + 1] = l[nt][e]; }
                     }
-                __threadfence();
                 __syncwarp();
-                // all consumer warps have published their partials -> one ticket for the CTA
+                // all consumer warps have written their partials (the barrier orders those stores
+                // before the one fence below) -> one ticket for the CTA
                 if (lane == 0) mbar_arrive(bar_seg);
-                if (!mbar_wait(bar_seg, seg_round & 1, s_abort)) break;
+                if (!mbar_wait(bar_seg, seg_round & 1, s_abort)) { alive = false; break; }
                 if (warp == 0 && lane == 0) {
+                    __threadfence();
                     const unsigned t = atomicAdd(&p.counters[seq], 1u);
                     const int last = (t == static_cast<unsigned>(n_seg - 1));
                     if (last) p.counters[seq] = 0;
+                    __threadfence();
                     *s_last = last;
                 }
                 if (lane == 0) mbar_arrive(bar_seg);
-                if (!mbar_wait(bar_seg, (seg_round + 1) & 1, s_abort)) break;
+                if (!mbar_wait(bar_seg, (seg_round + 1) & 1, s_abort)) { alive = false; break; }
                 seg_round += 2;
                 if (*s_last) {
-                    __threadfence();
                     merge_partials(p, seq, h, c_first, c_last, lane);
                 }
                 // the flag is rewritten only after every warp passed the next pair of barriers

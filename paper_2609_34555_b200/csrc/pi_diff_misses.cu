@@ -5,6 +5,7 @@
 //   misses     = selected blocks with block_table[b] < 0, ascending
 //   candidates = slots whose block is neither selected nor sink/local (free slots count),
 //                ordered by (stamp, slot) ascending; the i-th miss takes the i-th candidate
+//                (few misses: repeated block-wide arg-min; many: bitonic sort)
 //   update     = evicted block leaves the table, the miss enters it, every selected
 //                slot gets stamp = step
 //   list       = (block -> slot) pairs, runs that are consecutive on both sides merged
@@ -14,6 +15,8 @@ namespace {
 
 constexpr int DIFF_THREADS = 256;
 constexpr int DIFF_WARPS = DIFF_THREADS / 32;
+constexpr int ARGMIN_MAX_MISSES = 40;            // above this the full sort is cheaper
+constexpr int ARGMIN_KEYS_PER_THREAD = 4;        // register-resident keys: pools up to 1024 slots
 
 struct DiffParams {
     const int32_t* ctx_len;
@@ -60,6 +63,7 @@ diff_kernel(DiffParams p) {
     int32_t* s_miss = s_slot + p.K;                                                     // [K] j index of i-th miss
     unsigned char* s_used = reinterpret_cast<unsigned char*>(s_miss + p.K);             // [C] slot holds a selected block
     __shared__ int warp_tot[DIFF_WARPS];
+    __shared__ unsigned long long warp_min[2][DIFF_WARPS];
     __shared__ int s_ncand;
 
     const int seq = blockIdx.x, tid = threadIdx.x;
@@ -124,26 +128,56 @@ diff_kernel(DiffParams p) {
     const bool too_small = s_ncand < n_miss;
 
     if (n_miss > 0 && !too_small) {
-        // 3. bitonic sort of the candidate keys (ascending).  Warp w owns elements
-        // [32*E*w, 32*E*(w+1)), so exchanges at distance < 32*E stay inside one warp and need
-        // only a warp barrier; the few longer ones are fenced by CTA barriers.
-        const int E = max(1, p.Cpad / DIFF_THREADS), wspan = 32 * E;
-        const int lane = tid & 31, warp = tid >> 5;
-        for (int k = 2; k <= p.Cpad; k <<= 1) {
-            for (int j = k >> 1; j > 0; j >>= 1) {
-                if (j >= wspan) __syncthreads();
-                for (int e = 0; e < E; ++e) {
-                    const int i = (warp * E + e) * 32 + lane, l = i ^ j;
-                    if (l > i && l < p.Cpad) {
-                        const unsigned long long a = keys[i], b = keys[l];
-                        const bool up = (i & k) == 0;
-                        if ((a > b) == up) { keys[i] = b; keys[l] = a; }
-                    }
-                }
-                if (j >= wspan) __syncthreads(); else __syncwarp();
+        // 3. the n_miss smallest candidate keys, in order, end up in keys[0 .. n_miss).
+        if (n_miss <= ARGMIN_MAX_MISSES && p.Cpad <= DIFF_THREADS * ARGMIN_KEYS_PER_THREAD) {
+            // few misses (the steady state): n_miss rounds of a block-wide arg-min over keys held
+            // in registers, one CTA barrier per round (warp minima are double-buffered).
+            const int lane = tid & 31, warp = tid >> 5;
+            unsigned long long mine[ARGMIN_KEYS_PER_THREAD];
+#pragma unroll
+            for (int e = 0; e < ARGMIN_KEYS_PER_THREAD; ++e) {
+                const int s_ = tid + e * DIFF_THREADS;
+                mine[e] = s_ < p.Cpad ? keys[s_] : ~0ull;
             }
+            __syncthreads();                       // keys[] may now be overwritten with the result
+            for (int i = 0; i < n_miss; ++i) {
+                unsigned long long v = mine[0];
+#pragma unroll
+                for (int e = 1; e < ARGMIN_KEYS_PER_THREAD; ++e) v = min(v, mine[e]);
+#pragma unroll
+                for (int o = 16; o; o >>= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, o));
+                if (lane == 0) warp_min[i & 1][warp] = v;
+                __syncthreads();
+                unsigned long long g = warp_min[i & 1][0];
+#pragma unroll
+                for (int w = 1; w < DIFF_WARPS; ++w) g = min(g, warp_min[i & 1][w]);
+#pragma unroll
+                for (int e = 0; e < ARGMIN_KEYS_PER_THREAD; ++e)
+                    if (mine[e] == g) { mine[e] = ~0ull; keys[i] = g; }   // keys are unique (slot in the low word)
+            }
+            __syncthreads();
+        } else {
+            // many misses (cold start): bitonic sort of all candidate keys.  Warp w owns elements
+            // [32*E*w, 32*E*(w+1)), so exchanges at distance < 32*E stay inside one warp and need
+            // only a warp barrier; the few longer ones are fenced by CTA barriers.
+            const int E = max(1, p.Cpad / DIFF_THREADS), wspan = 32 * E;
+            const int lane = tid & 31, warp = tid >> 5;
+            for (int k = 2; k <= p.Cpad; k <<= 1) {
+                for (int j = k >> 1; j > 0; j >>= 1) {
+                    if (j >= wspan) __syncthreads();
+                    for (int e = 0; e < E; ++e) {
+                        const int i = (warp * E + e) * 32 + lane, l = i ^ j;
+                        if (l > i && l < p.Cpad) {
+                            const unsigned long long a = keys[i], b = keys[l];
+                            const bool up = (i & k) == 0;
+                            if ((a > b) == up) { keys[i] = b; keys[l] = a; }
+                        }
+                    }
+                    if (j >= wspan) __syncthreads(); else __syncwarp();
+                }
+            }
+            __syncthreads();
         }
-        __syncthreads();
         // 4. i-th miss takes the i-th candidate
         for (int i = tid; i < n_miss; i += DIFF_THREADS) {
             const int j = s_miss[i];
