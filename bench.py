@@ -127,6 +127,25 @@ def make_all_queries(cfg, steps: int, device) -> torch.Tensor:
     return torch.stack(per_layer, dim=1).contiguous()
 
 
+def rank_config(base, rank: int):
+    """Every rank runs the same shape on its own sequences: only the seed differs."""
+    return base.replace(seed=base.seed + 7919 * rank)
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    if world <= 1:
+        return ms
+    import torch.distributed as dist
+    tm = torch.tensor([ms], device=device)
+    dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+    return float(tm.item())
+
+
+def whole_job_value(world: int, steps: int, n_layers: int, ms: float) -> float:
+    """Layer-steps per second of the whole job: every rank did steps * n_layers of them."""
+    return world * steps * n_layers / (ms * 1e-3)
+
+
 def run_ours(args) -> dict:
     from paper_2609_34555_b200 import h2d_copy_ms
     from paper_2609_34555_b200.runner import StageTimer
@@ -141,7 +160,7 @@ def run_ours(args) -> dict:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     base = get_config(args.config)
-    cfg = base.replace(seed=base.seed + 7919 * rank)
+    cfg = rank_config(base, rank)
     if args.layers > 0:                       # profiling only: fewer layers of the same shape
         cfg = cfg.replace(n_layers=min(args.layers, cfg.n_layers), name=f"{cfg.name}[{args.layers} layers only]")
     K, W = args.steps, max(3, args.warmup)
@@ -189,12 +208,7 @@ def run_ours(args) -> dict:
     e1.record()
     barrier()
     clocks = sampler.stop()
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        import torch.distributed as dist
-        tm = torch.tensor([ms], device=dev)
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        ms = float(tm.item())
+    ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
     stats = pi.stats(reset=True)
     stages = timer.summary()
     status = pi.status()
@@ -226,14 +240,9 @@ def run_ours(args) -> dict:
             sess.decode_step_from_host(q_host[i], out_host, q_dev)
         a1.record()
         barrier()
-        e2e_ms = a0.elapsed_time(a1)
-        if world > 1:
-            import torch.distributed as dist
-            tm = torch.tensor([e2e_ms], device=dev)
-            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-            e2e_ms = float(tm.item())
+        e2e_ms = max_over_ranks(a0.elapsed_time(a1), world, dev)
         e2e_stats = pi.stats(reset=True)
-        e2e = dict(value=world * n_e2e * cfg.n_layers / (e2e_ms * 1e-3), unit="layer-steps/s",
+        e2e = dict(value=whole_job_value(world, n_e2e, cfg.n_layers, e2e_ms), unit="layer-steps/s",
                    h2d_bytes_per_step=int(q_dev.numel() * 2), d2h_bytes_per_step=int(out_host.numel() * 2),
                    misses_per_seq_layer_step=e2e_stats["missing_blocks"] / max(1, e2e_stats["sequences"]),
                    note="host KV store is read by the recall kernel in both forms")
@@ -252,7 +261,7 @@ def run_ours(args) -> dict:
     ser_recall_gbs = ser_stats["missing_blocks"] * cfg.block_bytes / max(1e-9, ser["recall"]["total_ms"] * 1e-3) / 1e9
     recall_gbs = recall_bytes / max(1e-9, recall_s) / 1e9
     line = {
-        "metric": METRIC, "value": world * K * cfg.n_layers / (ms * 1e-3), "unit": "layer-steps/s",
+        "metric": METRIC, "value": whole_job_value(world, K, cfg.n_layers, ms), "unit": "layer-steps/s",
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms / K, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{cfg.name}: {cfg.n_layers} layers x batch {cfg.batch} x ctx {cfg.ctx}, "

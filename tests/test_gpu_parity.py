@@ -60,3 +60,83 @@ def test_cold_start_empty_pool():
     case = make_case(cfg, steps=3, fill=0.0)                    # only sink/local resident
     stats = run_and_compare(case, steps=3)
     assert stats["extents"] < sum(stats["misses"])            # cold fill lands in adjacent slots: runs merge
+
+
+def test_cold_start_with_many_misses_takes_the_sort_path():
+    from tests.parity import make_case, run_and_compare
+    cfg = tiny_config(batch=2, ctx=16000, n_q_heads=16, n_kv_heads=4, budget_blocks=100, resident_frac=0.2)
+    case = make_case(cfg, steps=3, fill=0.0)                    # 91 misses per sequence at step 1
+    stats = run_and_compare(case, steps=3)
+    assert max(stats["misses"]) > 40 and min(stats["misses"]) <= 40
+
+
+def test_full_size_config2_shapes_sampled_sequences():
+    """Launch configuration of the bench (batch 16, 2048 blocks, K 128, C 409, pipelined
+    DecodeSession) on two of the 32 layers; the oracle follows three of the 16 sequences."""
+    from tests.parity import run_session_sampled
+    cfg = get_config("c2").replace(n_layers=2)
+    stats = run_session_sampled(cfg, steps=3, sample_seqs=[0, 7, 15])
+    assert stats["misses"] > 0
+
+
+def test_full_size_config4_shapes_group_of_eight_sampled():
+    """70B-shaped layer (64 query heads / 8 kv heads, 4096 blocks, K 256, C 614), one layer,
+    two of the 8 sequences followed by the oracle."""
+    from tests.parity import run_session_sampled
+    cfg = get_config("c4").replace(n_layers=1)
+    run_session_sampled(cfg, steps=2, sample_seqs=[1, 6])
+
+
+def gen_pinned(cfg):
+    from workloads import generate as gen
+    return gen.pinned_blocks(cfg).tolist()
+
+
+def test_errors_seen_on_the_device_or_at_the_boundary():
+    import paper_2609_34555_b200 as pkg
+    from paper_2609_34555_b200.runner import LayerBuffers
+    cfg = tiny_config(batch=2, ctx=1000)
+    dev = torch.device("cuda:0")
+    pi = pkg.PulseInfer.from_workload(cfg)
+    buf = LayerBuffers(pi, cfg.batch, dev)
+    # an unpinned host store is refused before anything is launched
+    host = torch.zeros((cfg.batch, cfg.n_blocks, cfg.block_bytes // 2), dtype=torch.bfloat16)
+    with pytest.raises(pkg.PiError) as e:
+        pi.recall_gather_scatter(0, host, buf.pool, buf.recall_list, buf.recall_count)
+    assert e.value.code == -5
+    # a selection index out of range sets the status word and is skipped, nothing faults
+    ctx = torch.full((cfg.batch,), cfg.ctx, dtype=torch.int32, device=dev)
+    buf.sel_blocks.fill_(-1)
+    buf.sel_blocks[0, 0] = 10 ** 6
+    buf.sel_count.fill_(1)
+    buf.sel_blocks[1, 0] = 0
+    pi.diff_misses(0, 1, ctx, buf.sel_blocks, buf.sel_count, buf.block_table, buf.slot_block, buf.slot_stamp,
+                   buf.sel_slots, buf.recall_list, buf.recall_count)
+    torch.cuda.synchronize()
+    st = pi.status()
+    assert st[0] == -8 and st[1] == 2 and st[2] == 0 and st[4] == 10 ** 6
+    assert buf.sel_slots[0, 0].item() == -1 and buf.recall_count[0].item() == 0
+    pi.clear_status()
+    assert pi.status()[0] == 0
+    # a pool with fewer evictable slots than misses: tables untouched, status says so
+    small = tiny_config(batch=1, ctx=1000, resident_frac=0.0)                    # C == K == 24
+    pi2 = pkg.PulseInfer.from_workload(small)
+    b2 = LayerBuffers(pi2, 1, dev)
+    C = small.pool_slots
+    pinned = gen_pinned(small)
+    middle = [b for b in range(small.n_blocks) if b not in set(pinned)]
+    res = torch.tensor([pinned + middle[:C - len(pinned)]], dtype=torch.int32, device=dev)
+    pi2.table_init(res, b2.block_table, b2.slot_block, b2.slot_stamp)
+    sel = torch.tensor([middle[C:C + small.budget_blocks]], dtype=torch.int32, device=dev)    # 24 misses, 15 candidates
+    cnt = torch.tensor([small.budget_blocks], dtype=torch.int32, device=dev)
+    ctx1 = torch.tensor([small.ctx], dtype=torch.int32, device=dev)
+    before = (b2.block_table.clone(), b2.slot_block.clone(), b2.slot_stamp.clone())
+    pi2.diff_misses(0, 3, ctx1, sel, cnt, b2.block_table, b2.slot_block, b2.slot_stamp, b2.sel_slots,
+                    b2.recall_list, b2.recall_count)
+    torch.cuda.synchronize()
+    st = pi2.status()
+    assert st[0] == -4 and st[1] == 2 and st[3] == small.budget_blocks and st[4] == C - len(pinned)
+    assert b2.recall_count[0].item() == 0 and (b2.sel_slots == -1).all()
+    assert all(torch.equal(a, b) for a, b in zip(before, (b2.block_table, b2.slot_block, b2.slot_stamp)))
+    pi2.close()
+    pi.close()
