@@ -96,7 +96,7 @@ class ClockSampler:
                     samples=len(sm), reasons=sorted(reasons))
 
 
-def build_session(cfg, rank: int, host_layers_arg: int, world: int):
+def build_session(cfg, rank: int, host_layers_arg: int, world: int, recall_ctas: int = 0):
     from paper_2609_34555_b200 import PulseInfer
     from paper_2609_34555_b200.runner import DecodeSession
     from workloads import generate as gen
@@ -107,7 +107,7 @@ def build_session(cfg, rank: int, host_layers_arg: int, world: int):
     else:
         budget = 0.55 * mem_available_bytes() / max(1, world)
         R = int(max(1, min(cfg.n_layers, budget // per_layer)))
-    pi = PulseInfer.from_workload(cfg)
+    pi = PulseInfer.from_workload(cfg, recall_ctas=recall_ctas)
     sess = DecodeSession(pi, cfg.batch, cfg.n_layers, host_layers=R)
     sess.ctx_len.fill_(cfg.ctx)
     dev = sess.device
@@ -166,7 +166,7 @@ def run_ours(args) -> dict:
     K, W = args.steps, max(3, args.warmup)
 
     t_setup = time.time()
-    pi, sess, R = build_session(cfg, rank, args.host_layers, world)
+    pi, sess, R = build_session(cfg, rank, args.host_layers, world, args.recall_ctas)
     n_e2e = K if not args.no_e2e else 0
     n_serial = min(K, 4)
     q_all = make_all_queries(cfg, args.settle + W + K + n_serial + n_e2e, dev)
@@ -402,6 +402,7 @@ def main():
     ap.add_argument("--host-layers", type=int, default=0, help="distinct host KV regions (0 = as many as fit)")
     ap.add_argument("--settle", type=int, default=24, help="untimed decode steps before the warm-up")
     ap.add_argument("--layers", type=int, default=0, help="cut the layer stack (for profiler captures only)")
+    ap.add_argument("--recall-ctas", type=int, default=0, help="CTAs of the recall kernel (0 = library default)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)

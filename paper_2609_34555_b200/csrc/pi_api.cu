@@ -57,7 +57,8 @@ extern "C" int pi_create(const pi_config* cfg, pi_ctx** out) {
     if (e != cudaSuccess) { (void)cudaGetLastError(); pi_destroy(c); return PI_ERR_CUDA; }
     c->n_sms = prop.multiProcessorCount;
     c->attn_ctas = cfg->attn_ctas > 0 ? cfg->attn_ctas : c->n_sms;
-    c->recall_ctas = cfg->recall_ctas > 0 ? cfg->recall_ctas : 32;
+    // ten CTAs (80 warps x 4 KB in flight) saturate the host link on a B200; more only queue requests up
+    c->recall_ctas = cfg->recall_ctas > 0 ? cfg->recall_ctas : 10;
 
     const size_t nb = static_cast<size_t>(cfg->max_batch);
     const size_t n_part = static_cast<size_t>(c->attn_ctas) + nb;

@@ -8,8 +8,9 @@
 // tiled TMA loads (128-byte swizzle, no multicast); consumer warp h computes, for its
 // G query heads,  S^T = K q^T  (tokens on M, heads on N, bf16 mma, fp32 accumulate),
 // an online softmax over tokens, and  O^T += V^T P.  A (CTA, sequence) segment that
-// does not cover its whole sequence writes an fp32 partial (m, l, O); the CTA whose
-// ticket completes the sequence merges the partials.  No CTA waits for another.
+// does not cover its whole sequence writes an fp32 partial (m, l, O); a small second
+// kernel, launched with programmatic stream serialization so that its start-up overlaps
+// this kernel's tail, merges the partials.  No CTA waits for another.
 //
 // The arithmetic intensity is G flop per byte: HBM-bound by a wide margin, so the
 // design goal is bytes in flight (ring of Hkv*8 KB stages), not tensor throughput.
@@ -113,94 +114,102 @@ __device__ __forceinline__ int seq_of_unit(const int* pref, int batch, int u) {
     return lo;
 }
 
-// Merge of the split-K partials of one sequence by warp h for its G query heads.  Lane i
-// fetches (m, l) of segment i once, the warp agrees on the maximum, and the weighted sum of
-// the partial outputs runs over segments with sixteen independent 16-byte loads in flight per
-// lane (4 heads x 4 segments), the first batch issued before the weights are known; each lane
-// owns 4 of the 128 channels.
-__device__ __forceinline__ void merge_partials(const AttnParams& p, int seq, int h, int c_first, int c_last, int lane) {
+// Second kernel of the attention call: merges the split-K partials of every sequence that
+// was cut across CTAs.  Grid (Hkv, batch), one warp per query head, lane = 4 channels.  It is
+// launched with programmatic stream serialization: its CTAs may start while the main kernel
+// still runs, work out which partials belong to their sequence (same split arithmetic as the
+// main kernel), and only then wait for the main grid to complete and flush.
+__global__ void __launch_bounds__(512)
+attn_merge_kernel(AttnParams p, int main_ctas) {
+    __shared__ int s_red[3][16];
+    const int seq = blockIdx.y, h = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    const int SUB = p.B >> 4;
+    // units before this sequence, of this sequence, and in total
+    int before = 0, mine = 0, total = 0;
+    for (int s = threadIdx.x; s < p.batch; s += blockDim.x) {
+        int n = p.sel_count[s];
+        if (n < 0 || n > p.K) n = 0;
+        n *= SUB;
+        total += n;
+        if (s < seq) before += n;
+        if (s == seq) mine = n;
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+        before += __shfl_xor_sync(0xffffffffu, before, o);
+        mine += __shfl_xor_sync(0xffffffffu, mine, o);
+        total += __shfl_xor_sync(0xffffffffu, total, o);
+    }
+    if (lane == 0) { s_red[0][warp] = before; s_red[1][warp] = mine; s_red[2][warp] = total; }
+    __syncthreads();
+    before = mine = total = 0;
+    for (int w = 0; w < n_warps; ++w) { before += s_red[0][w]; mine += s_red[1][w]; total += s_red[2][w]; }
+    if (mine == 0) return;                                    // nothing selected: the main kernel wrote zeros
+    const long long U = total, P = min(static_cast<long long>(main_ctas), max(U, 1ll));
+    const int c_first = cta_of_unit(before, U, P), c_last = cta_of_unit(before + mine - 1, U, P);
     const int n_seg = c_last - c_first + 1;
+    if (n_seg == 1) return;                                   // one CTA covered the sequence and wrote the result
+
+    asm volatile("griddepcontrol.wait;" ::: "memory");        // main grid complete, its stores visible
+
     const size_t slot0 = static_cast<size_t>(c_first) + seq;
-    for (int g0 = 0; g0 < p.G; g0 += 4) {
-        const size_t head0 = static_cast<size_t>(h) * p.G + g0;
-        float M[4], L[4];
-        float4 acc[4];
-#pragma unroll
-        for (int gi = 0; gi < 4; ++gi) { M[gi] = -INFINITY; L[gi] = 0.f; acc[gi] = make_float4(0.f, 0.f, 0.f, 0.f); }
-        // pass 1: maxima (one load per lane per head when n_seg <= 32)
-        float2 ml0[4];
-#pragma unroll
-        for (int gi = 0; gi < 4; ++gi) ml0[gi] = make_float2(-INFINITY, 0.f);
-        for (int s0 = 0; s0 < n_seg; s0 += 32) {
-            const int sg = s0 + lane;
-#pragma unroll
-            for (int gi = 0; gi < 4; ++gi)
-                if (sg < n_seg && g0 + gi < p.G) {
-                    const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((slot0 + sg) * p.Hq + head0 + gi) * 2));
-                    if (s0 == 0) ml0[gi] = ml;
-                    M[gi] = fmaxf(M[gi], ml.x);
-                }
+    for (int g = warp; g < p.G; g += n_warps) {
+        const size_t head = static_cast<size_t>(h) * p.G + g;
+        // lane i holds (m, l) of segment i (+32, +64, ...).  The first eight partial outputs are
+        // requested in the same breath (they do not depend on the weights), so a sequence cut into
+        // up to eight segments costs one round trip to L2.
+        float2 ml0 = make_float2(-INFINITY, 0.f);
+        float M = -INFINITY;
+        for (int sg = lane; sg < n_seg; sg += 32) {
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((slot0 + sg) * p.Hq + head) * 2));
+            if (sg < 32) ml0 = ml;
+            M = fmaxf(M, ml.x);
         }
-        // first batch of partial outputs: independent of the weights, so issued before the reduction
-        float4 v[4][4];
-        auto fetch = [&](int base_seg) {
+        float4 v[8];
+        auto fetch = [&](int first) {
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-#pragma unroll
-                for (int gi = 0; gi < 4; ++gi) {
-                    v[kk][gi] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (base_seg + kk < n_seg && g0 + gi < p.G)
-                        v[kk][gi] = __ldcg(reinterpret_cast<const float4*>(
-                                        p.part_o + ((slot0 + base_seg + kk) * p.Hq + head0 + gi) * PI_HEAD_DIM) + lane);
-                }
+            for (int kk = 0; kk < 8; ++kk) {
+                v[kk] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (first + kk < n_seg)
+                    v[kk] = __ldcg(reinterpret_cast<const float4*>(p.part_o + ((slot0 + first + kk) * p.Hq + head) * PI_HEAD_DIM) + lane);
+            }
         };
         fetch(0);
 #pragma unroll
-        for (int gi = 0; gi < 4; ++gi)
-#pragma unroll
-            for (int o = 16; o; o >>= 1) M[gi] = fmaxf(M[gi], __shfl_xor_sync(0xffffffffu, M[gi], o));
+        for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float L = 0.f;
         for (int s0 = 0; s0 < n_seg; s0 += 32) {
             const int sg = s0 + lane;
-            float w[4];
-#pragma unroll
-            for (int gi = 0; gi < 4; ++gi) {
-                w[gi] = 0.f;
-                if (sg < n_seg && g0 + gi < p.G) {
-                    const float2 ml = s0 == 0 ? ml0[gi]
-                        : __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((slot0 + sg) * p.Hq + head0 + gi) * 2));
-                    w[gi] = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M[gi]);
-                    L[gi] += w[gi] * ml.y;
-                }
+            float w = 0.f;
+            if (sg < n_seg) {
+                const float2 ml = s0 == 0 ? ml0
+                    : __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((slot0 + sg) * p.Hq + head) * 2));
+                w = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M);
+                L += w * ml.y;
             }
             const int cnt = min(32, n_seg - s0);
-            for (int k = 0; k < cnt; k += 4) {
+            for (int k = 0; k < cnt; k += 8) {
                 if (s0 + k > 0) fetch(s0 + k);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-#pragma unroll
-                    for (int gi = 0; gi < 4; ++gi) {
-                        const float wk = __shfl_sync(0xffffffffu, w[gi], (k + kk) & 31);
-                        acc[gi].x += wk * v[kk][gi].x; acc[gi].y += wk * v[kk][gi].y;
-                        acc[gi].z += wk * v[kk][gi].z; acc[gi].w += wk * v[kk][gi].w;
-                    }
+                for (int kk = 0; kk < 8; ++kk) {
+                    const float wk = __shfl_sync(0xffffffffu, w, (k + kk) & 31);
+                    acc.x += wk * v[kk].x; acc.y += wk * v[kk].y; acc.z += wk * v[kk].z; acc.w += wk * v[kk].w;
+                }
             }
         }
 #pragma unroll
-        for (int gi = 0; gi < 4; ++gi) {
-#pragma unroll
-            for (int o = 16; o; o >>= 1) L[gi] += __shfl_xor_sync(0xffffffffu, L[gi], o);
-            if (g0 + gi >= p.G) continue;
-            const float inv = L[gi] > 0.f ? 1.f / L[gi] : 0.f;
-            const size_t gh = static_cast<size_t>(seq) * p.Hq + head0 + gi;
-            __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc[gi].x * inv, acc[gi].y * inv);
-            __nv_bfloat162 hi2 = __floats2bfloat162_rn(acc[gi].z * inv, acc[gi].w * inv);
-            uint2 pk;
-            pk.x = *reinterpret_cast<uint32_t*>(&lo2);
-            pk.y = *reinterpret_cast<uint32_t*>(&hi2);
-            *reinterpret_cast<uint2*>(p.out + gh * PI_HEAD_DIM + lane * 4) = pk;
-            if (p.lse && lane == 0)
-                p.lse[gh] = L[gi] > 0.f ? (M[gi] + log2f(L[gi])) * 0.6931471805599453f : -INFINITY;
-        }
+        for (int o = 16; o; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+        const float inv = L > 0.f ? 1.f / L : 0.f;
+        const size_t gh = static_cast<size_t>(seq) * p.Hq + head;
+        __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+        __nv_bfloat162 hi2 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+        uint2 pk;
+        pk.x = *reinterpret_cast<uint32_t*>(&lo2);
+        pk.y = *reinterpret_cast<uint32_t*>(&hi2);
+        *reinterpret_cast<uint2*>(p.out + gh * PI_HEAD_DIM + lane * 4) = pk;
+        if (p.lse && lane == 0) p.lse[gh] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
     }
 }
 
@@ -219,9 +228,11 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
     int2* s_meta = reinterpret_cast<int2*>(s_last + 1);                                // [ATTN_META_UNITS] {slot row, sub*16 | nvalid<<8}
     int* s_pref = reinterpret_cast<int*>(s_meta + ATTN_META_UNITS);                    // [batch + 1]
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + ATTN_MAX_STAGES);
-    const uint32_t bar_seg = smem_u32(bars + 2 * ATTN_MAX_STAGES);
     const int SUB = p.B >> 4;
     if (tid == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&pool_map) : "memory");
+    // the merge kernel that follows in the stream may be scheduled from now on; it waits for this
+    // grid to finish before it reads anything this grid writes
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---- unit prefix over sequences (every CTA computes the same table)
     for (int s = tid; s < p.batch; s += blockDim.x) {
@@ -239,7 +250,6 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
             mbar_init(bar_full + 8 * i, 1);
             mbar_init(bar_empty + 8 * i, p.Hkv);
         }
-        mbar_init(bar_seg, p.Hkv);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -318,7 +328,6 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
     const int h = warp;
     const int row = lane >> 2, colp = (lane & 3) * 2;
     int seq = seq_of_unit(s_pref, p.batch, u0);
-    int seg_round = 0;
     // per-lane ldmatrix offsets inside a stage (swizzled 128-byte rows)
     const int r8 = lane & 7, mi = lane >> 3;
     const int tK = r8 + 8 * (mi & 1), cK = mi >> 1;         // K as A operand (rows = tokens)
@@ -465,26 +474,6 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
                         }
                         if (row == 0) { p.part_ml[gh * 2] = m[nt][e]; p.part_ml[gh * 2 + 1] = l[nt][e]; }
                     }
-                __syncwarp();
-                // all consumer warps have written their partials (the barrier orders those stores
-                // before the one fence below) -> one ticket for the CTA
-                if (lane == 0) mbar_arrive(bar_seg);
-                if (!mbar_wait(bar_seg, seg_round & 1, s_abort)) { alive = false; break; }
-                if (warp == 0 && lane == 0) {
-                    __threadfence();
-                    const unsigned t = atomicAdd(&p.counters[seq], 1u);
-                    const int last = (t == static_cast<unsigned>(n_seg - 1));
-                    if (last) p.counters[seq] = 0;
-                    __threadfence();
-                    *s_last = last;
-                }
-                if (lane == 0) mbar_arrive(bar_seg);
-                if (!mbar_wait(bar_seg, (seg_round + 1) & 1, s_abort)) { alive = false; break; }
-                seg_round += 2;
-                if (*s_last) {
-                    merge_partials(p, seq, h, c_first, c_last, lane);
-                }
-                // the flag is rewritten only after every warp passed the next pair of barriers
             }
         }
     }
@@ -540,6 +529,19 @@ int pi_launch_attn(pi_ctx* c, int batch, const void* q, const void* pool, const 
         PI_CUDA_TRY(cudaFuncSetAttribute(attn_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
         attn_kernel<2><<<c->attn_ctas, threads, smem, stream>>>(c->pool_map, p);
     }
+    PI_CUDA_TRY(cudaGetLastError());
+    // merge of the split sequences: may start early, synchronises on the grid above by itself
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(cfg.n_kv_heads, batch);
+    lc.blockDim = dim3(32 * (p.G < 16 ? p.G : 16));
+    lc.dynamicSmemBytes = 0;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    PI_CUDA_TRY(cudaLaunchKernelEx(&lc, attn_merge_kernel, p, c->attn_ctas));
     PI_CUDA_TRY(cudaGetLastError());
     return PI_OK;
 }

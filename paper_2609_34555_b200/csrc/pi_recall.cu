@@ -2,7 +2,9 @@
 // with wide loads and writes them into their pool slots.
 //
 // A small, fixed number of persistent CTAs (sized for the host link, not for the miss
-// count) walks one flat space of 4 KB pieces covering every extent of every list.
+// count: requests beyond what the link can absorb only queue up in the memory system and
+// slow the HBM traffic of kernels running beside this one) walks one flat space of 4 KB
+// pieces covering every extent of every list.
 // Lists and counts are read from device memory, so the kernel can be enqueued right
 // behind the diff kernel without a host round trip.  Neighbouring warps take
 // neighbouring pieces, so an extent of merged units is read as one long sequential
@@ -15,6 +17,10 @@ constexpr int RECALL_THREADS = 256;
 constexpr int RECALL_WARPS = RECALL_THREADS / 32;
 constexpr int PIECE_BYTES = 4096;                 // per warp per iteration: 8 x 16 B per lane
 constexpr int LOADS_PER_LANE = PIECE_BYTES / (32 * 16);
+// Extents cached in shared memory.  Kept to 12 KB on purpose: the attention kernel that runs
+// beside this one leaves about 20 KB of an SM's shared memory free, and a recall CTA that
+// does not fit next to an attention CTA costs the attention kernel a whole extra wave.
+constexpr int RECALL_CACHE_EXTENTS = 768;
 
 struct RecallParams {
     const unsigned char* host;
@@ -23,7 +29,7 @@ struct RecallParams {
     const int32_t* count;
     pi_status_ref st;
     long long host_stride, pool_stride, unit_bytes;
-    int n_lists, lists_per_seq, cap;
+    int n_lists, lists_per_seq, cap, cache_cap;
 };
 
 __device__ __forceinline__ uint4 ld_host16(const void* p) {
@@ -33,47 +39,89 @@ __device__ __forceinline__ uint4 ld_host16(const void* p) {
     return v;
 }
 
+// Block-wide exclusive scan of one value per thread over RECALL_THREADS threads, continued
+// from `run` (updated to the new running total).  All threads must call.
+__device__ __forceinline__ long long block_scan_add(long long v, long long* warp_tot, long long& run) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    long long inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        long long t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    __syncthreads();
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    long long base = run, tot = 0;
+#pragma unroll
+    for (int i = 0; i < RECALL_WARPS; ++i) {
+        if (i < warp) base += warp_tot[i];
+        tot += warp_tot[i];
+    }
+    run += tot;
+    return base + inc - v;
+}
+
 __global__ void __launch_bounds__(RECALL_THREADS)
 recall_kernel(RecallParams p) {
-    extern __shared__ long long s_pref[];          // [n_lists + 1] exclusive prefix of units per list
+    extern __shared__ long long s_dyn[];
+    long long* s_pref = s_dyn;                                  // [n_lists + 1] units before each list
+    int* s_eoff = reinterpret_cast<int*>(s_pref + p.n_lists + 1);      // [n_lists + 1] extents before each list
+    pi_extent* s_ext = reinterpret_cast<pi_extent*>(s_pref + p.n_lists + 1 + (p.n_lists + 2) / 2);   // [cache_cap]
     __shared__ long long warp_tot[RECALL_WARPS];
-    __shared__ long long s_run;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    // units per list = units_before + n_units of its last extent; prefix over lists
-    if (tid == 0) s_run = 0;
-    __syncthreads();
+    // 1. extents before each list (counts are validated once, here)
+    long long run = 0;
     for (int l0 = 0; l0 < p.n_lists; l0 += RECALL_THREADS) {
         const int l = l0 + tid;
-        long long u = 0;
+        int n = 0;
         if (l < p.n_lists) {
-            int n = p.count[l];
+            n = p.count[l];
             if (n < 0 || n > p.cap) {
                 if (blockIdx.x == 0) pi_report(p.st, PI_ERR_CAPACITY, PI_STAGE_RECALL, l, n, p.cap);
                 n = 0;
             }
+        }
+        const long long off = block_scan_add(n, warp_tot, run);
+        if (l < p.n_lists) s_eoff[l] = static_cast<int>(off);
+    }
+    if (tid == 0) s_eoff[p.n_lists] = static_cast<int>(run);
+    __syncthreads();
+    const int n_ext = s_eoff[p.n_lists];
+    const bool cached = n_ext <= p.cache_cap;
+
+    // 2. all extents into shared memory in one round of loads (when they fit), so that finding
+    //    a piece's extent later costs no global round trip
+    if (cached) {
+        for (int i = tid; i < n_ext; i += RECALL_THREADS) {
+            int lo = 0, hi = p.n_lists;                          // last l with s_eoff[l] <= i
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (s_eoff[mid] <= i) lo = mid; else hi = mid;
+            }
+            s_ext[i] = p.list[static_cast<size_t>(lo) * p.cap + (i - s_eoff[lo])];
+        }
+        __syncthreads();
+    }
+
+    // 3. units before each list: a list's total is units_before + n_units of its last extent
+    run = 0;
+    for (int l0 = 0; l0 < p.n_lists; l0 += RECALL_THREADS) {
+        const int l = l0 + tid;
+        long long u = 0;
+        if (l < p.n_lists) {
+            const int n = s_eoff[l + 1] - s_eoff[l];
             if (n > 0) {
-                const pi_extent e = p.list[static_cast<size_t>(l) * p.cap + n - 1];
+                const pi_extent e = cached ? s_ext[s_eoff[l + 1] - 1] : p.list[static_cast<size_t>(l) * p.cap + n - 1];
                 u = static_cast<long long>(e.units_before) + e.n_units;
                 if (u < 0) u = 0;
             }
         }
-        long long inc = u;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            long long t = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += t;
-        }
-        if (lane == 31) warp_tot[warp] = inc;
-        __syncthreads();
-        long long base = s_run;
-        for (int i = 0; i < warp; ++i) base += warp_tot[i];
-        if (l < p.n_lists) s_pref[l] = base + inc - u;
-        __syncthreads();
-        if (tid == RECALL_THREADS - 1) s_run = base + inc;
-        __syncthreads();
+        const long long off = block_scan_add(u, warp_tot, run);
+        if (l < p.n_lists) s_pref[l] = off;
     }
-    if (tid == 0) s_pref[p.n_lists] = s_run;
+    if (tid == 0) s_pref[p.n_lists] = run;
     __syncthreads();
 
     const long long pieces_per_unit = p.unit_bytes / PIECE_BYTES;
@@ -91,8 +139,8 @@ recall_kernel(RecallParams p) {
         const int l = lo;
         const int u_in_list = static_cast<int>(unit - s_pref[l]);
         // extent inside the list: last e with units_before <= u_in_list
-        const pi_extent* ext = p.list + static_cast<size_t>(l) * p.cap;
-        int elo = 0, ehi = p.count[l];
+        const pi_extent* ext = cached ? s_ext + s_eoff[l] : p.list + static_cast<size_t>(l) * p.cap;
+        int elo = 0, ehi = s_eoff[l + 1] - s_eoff[l];
         while (ehi - elo > 1) {
             const int mid = (elo + ehi) >> 1;
             if (ext[mid].units_before <= u_in_list) elo = mid; else ehi = mid;
@@ -126,9 +174,19 @@ int pi_launch_recall(pi_ctx* c, int n_lists, int lists_per_seq, const void* host
     p.st = pi_status_of(c);
     p.host_stride = host_stride; p.pool_stride = pool_stride; p.unit_bytes = unit_bytes;
     p.n_lists = n_lists; p.lists_per_seq = lists_per_seq; p.cap = cap;
-    const size_t smem = (static_cast<size_t>(n_lists) + 1) * sizeof(long long);
+    // shared memory: two prefix arrays over the lists + the extent cache
+    const long long want = static_cast<long long>(n_lists) * cap;
+    p.cache_cap = static_cast<int>(want < RECALL_CACHE_EXTENTS ? want : RECALL_CACHE_EXTENTS);
+    const size_t smem = (static_cast<size_t>(n_lists) + 1) * sizeof(long long) +
+                        ((static_cast<size_t>(n_lists) + 2) / 2) * sizeof(long long) +
+                        static_cast<size_t>(p.cache_cap) * sizeof(pi_extent);
     if (smem > 40 * 1024)
         PI_CUDA_TRY(cudaFuncSetAttribute(recall_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    // ask for the largest shared-memory carve-out although this kernel hardly uses any: an SM
+    // keeps one L1/shared split for all resident CTAs, and the attention kernel that overlaps
+    // this one needs nearly all of it -- with the default split its CTAs could not join ours
+    PI_CUDA_TRY(cudaFuncSetAttribute(recall_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                     cudaSharedmemCarveoutMaxShared));
     recall_kernel<<<c->recall_ctas, RECALL_THREADS, smem, stream>>>(p);
     PI_CUDA_TRY(cudaGetLastError());
     return PI_OK;

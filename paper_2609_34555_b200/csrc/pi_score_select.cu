@@ -37,6 +37,7 @@ struct SelParams {
     unsigned int* counters;
     pi_status_ref st;
     int h_star, Hq, G, B, K, n_sink, n_local, max_blocks;
+    int batch, per;                                // sequences in the launch, chunks per CTA
 };
 
 // Shared arrays that one thread walks with a stride of several words are stored with one
@@ -92,111 +93,16 @@ __device__ __forceinline__ unsigned block_excl_scan(unsigned v, unsigned* warp_t
     return base + inc - v;
 }
 
-__global__ void __launch_bounds__(SCORE_THREADS, 2)
-score_select_kernel(SelParams p) {
-    extern __shared__ uint32_t keys[];             // [padded(n_blocks)] in the selecting CTA
-    __shared__ unsigned hist[BINS + BINS / 32 + 1];
-    __shared__ unsigned warp_tot[SCORE_WARPS];
-    __shared__ uint32_t red_lo[SCORE_WARPS], red_hi[SCORE_WARPS];
-    __shared__ uint32_t cand_key[RESOLVE_MAX];
-    __shared__ int cand_idx[RESOLVE_MAX];
-    __shared__ uint32_t sh_lo, sh_hi;
-    __shared__ unsigned sh_need, sh_cnt, sh_ncand;
-    __shared__ int sh_last;
+struct SelShared {
+    uint32_t lo, hi;
+    unsigned need, cnt, ncand;
+};
 
-    const int seq = blockIdx.y;
+// Selection for one sequence by the whole CTA, from the fp32 scores in global memory.
+__device__ __forceinline__ void select_sequence(const SelParams& p, int seq, int n_blocks, uint32_t* keys, unsigned* hist,
+                                                unsigned* warp_tot, uint32_t* red_lo, uint32_t* red_hi,
+                                                uint32_t* cand_key, int* cand_idx, SelShared& sh) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-    // ---------------- phase 1: scores of this CTA's chunk.  Every load (digest rows, the
-    // group's queries, the context length) is issued before anything waits: digest rows up
-    // to max_blocks are allocated, so they are read unguarded and masked at the store.
-    const int b0 = blockIdx.x * SCORE_CHUNK + warp * BLOCKS_PER_WARP;
-    const uint4* dg = p.digest + static_cast<size_t>(seq) * p.max_blocks * 32;   // 32 uint4 per block
-    uint4 v[BLOCKS_PER_WARP];
-#pragma unroll
-    for (int i = 0; i < BLOCKS_PER_WARP; ++i) {
-        v[i] = make_uint4(0, 0, 0, 0);
-        if (b0 + i < p.max_blocks) v[i] = ld_stream16(dg + static_cast<size_t>(b0 + i) * 32 + lane);
-    }
-    // lanes 0-15 hold Q- for channels 8*lane.., lanes 16-31 hold Q+ for channels 8*(lane-16)..
-    float w[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) w[i] = 0.f;
-    {
-        const int d0 = (lane & 15) * 8;
-        const bool plus = lane >= 16;
-        const __nv_bfloat16* qh = p.q + (static_cast<size_t>(seq) * p.Hq + static_cast<size_t>(p.h_star) * p.G) * PI_HEAD_DIM + d0;
-        // the group's query rows are fetched four at a time so their latencies overlap
-        for (int g0 = 0; g0 < p.G; g0 += 4) {
-            uint4 qv[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                qv[j] = make_uint4(0, 0, 0, 0);
-                if (g0 + j < p.G) qv[j] = *reinterpret_cast<const uint4*>(qh + static_cast<size_t>(g0 + j) * PI_HEAD_DIM);
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&qv[j]);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    float2 f = __bfloat1622float2(h2[i]);
-                    w[2 * i] += plus ? fmaxf(f.x, 0.f) : fminf(f.x, 0.f);
-                    w[2 * i + 1] += plus ? fmaxf(f.y, 0.f) : fminf(f.y, 0.f);
-                }
-            }
-        }
-    }
-    int ctx = p.ctx_len[seq];
-    if (ctx < 0) ctx = 0;
-    int n_blocks = (ctx + p.B - 1) / p.B;
-    if (n_blocks > p.max_blocks) {
-        if (tid == 0 && blockIdx.x == 0) pi_report(p.st, PI_ERR_CAPACITY, PI_STAGE_SELECT, seq, n_blocks, p.max_blocks);
-        n_blocks = p.max_blocks;
-    }
-    {
-        float s[BLOCKS_PER_WARP];
-#pragma unroll
-        for (int i = 0; i < BLOCKS_PER_WARP; ++i) s[i] = dot8(v[i], w);
-        // transposed warp reduction: 8 values x 32 lanes -> lane group (lane>>2) owns block (lane>>2)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const bool up = lane & 16;
-            float send = up ? s[i] : s[i + 4];
-            float keep = up ? s[i + 4] : s[i];
-            s[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
-        }
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            const bool up = lane & 8;
-            float send = up ? s[i] : s[i + 2];
-            float keep = up ? s[i + 2] : s[i];
-            s[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
-        }
-        {
-            const bool up = lane & 4;
-            float send = up ? s[0] : s[1];
-            float keep = up ? s[1] : s[0];
-            s[0] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-        }
-        s[0] += __shfl_xor_sync(0xffffffffu, s[0], 2);
-        s[0] += __shfl_xor_sync(0xffffffffu, s[0], 1);
-        const int b = b0 + (lane >> 2);
-        if ((lane & 3) == 0 && b < n_blocks) p.scores[static_cast<size_t>(seq) * p.max_blocks + b] = s[0];
-    }
-
-    // ---------------- ticket: the last CTA of the sequence selects
-    // (the CTA barrier orders every thread's score stores before thread 0's fence and ticket)
-    __syncthreads();
-    if (tid == 0) {
-        __threadfence();
-        unsigned t = atomicAdd(&p.counters[seq], 1u);
-        sh_last = (t == gridDim.x - 1);
-        if (sh_last) p.counters[seq] = 0;           // ready for the next launch
-        __threadfence();
-    }
-    __syncthreads();
-    if (!sh_last) return;
-
     // ---------------- phase 2: selection
     const int m_lo = min(p.n_sink, n_blocks);
     const int m_hi = max(n_blocks - p.n_local, m_lo);
@@ -206,6 +112,7 @@ score_select_kernel(SelParams p) {
 
     uint32_t kmin = 0xffffffffu, kmax = 0u;
     const float* sc = p.scores + static_cast<size_t>(seq) * p.max_blocks;
+    for (int i = tid; i < BINS + BINS / 32 + 1; i += SCORE_THREADS) hist[i] = 0;   // overlaps the key loads below
     for (int i = tid; i < n_blocks; i += SCORE_THREADS) {
         uint32_t key = float_key(__ldcg(sc + i));
         keys[padded(i)] = key;
@@ -235,8 +142,10 @@ score_select_kernel(SelParams p) {
             if (range == 0) break;                   // every key left is equal: ties by index
             const int bits = 32 - __clz(range);
             const int shift = bits > 11 ? bits - 11 : 0;
-            for (int i = tid; i < BINS + BINS / 32 + 1; i += SCORE_THREADS) hist[i] = 0;
-            __syncthreads();
+            if (pass > 0) {                          // the first pass finds the histogram already cleared
+                for (int i = tid; i < BINS + BINS / 32 + 1; i += SCORE_THREADS) hist[i] = 0;
+                __syncthreads();
+            }
             for (int i = m_lo + tid; i < m_hi; i += SCORE_THREADS) {
                 const uint32_t key = keys[padded(i)];
                 if (key >= lo && key <= hi) atomicAdd(&hist[padded((key - lo) >> shift)], 1u);
@@ -256,25 +165,25 @@ score_select_kernel(SelParams p) {
                     if (need > acc && need <= acc + hb[j]) {
                         const uint32_t nlo = lo + (static_cast<uint32_t>(top - j) << shift);
                         const uint32_t span = shift ? ((1u << shift) - 1u) : 0u;
-                        sh_lo = nlo;
-                        sh_hi = (hi - nlo < span) ? hi : nlo + span;
-                        sh_need = need - acc;
-                        sh_cnt = hb[j];
+                        sh.lo = nlo;
+                        sh.hi = (hi - nlo < span) ? hi : nlo + span;
+                        sh.need = need - acc;
+                        sh.cnt = hb[j];
                     }
                     acc += hb[j];
                 }
-                sh_ncand = 0;
+                sh.ncand = 0;
             }
             __syncthreads();
-            lo = sh_lo; hi = sh_hi; need = sh_need;
-            const unsigned cnt = sh_cnt;
+            lo = sh.lo; hi = sh.hi; need = sh.need;
+            const unsigned cnt = sh.cnt;
             if (shift == 0 || cnt == need) break;
             if (cnt <= RESOLVE_MAX) {
                 // few keys left in the bucket: one warp ranks them by (key descending, index ascending)
                 for (int i = m_lo + tid; i < m_hi; i += SCORE_THREADS) {
                     const uint32_t key = keys[padded(i)];
                     if (key >= lo && key <= hi) {
-                        const unsigned pos = atomicAdd(&sh_ncand, 1u);
+                        const unsigned pos = atomicAdd(&sh.ncand, 1u);
                         cand_key[pos] = key;
                         cand_idx[pos] = i;
                     }
@@ -294,10 +203,10 @@ score_select_kernel(SelParams p) {
                     const unsigned is_tau = __ballot_sync(0xffffffffu, have && rank == need - 1);
                     const uint32_t tau = __shfl_sync(0xffffffffu, mk, __ffs(is_tau) - 1);
                     const unsigned eq_taken = __popc(__ballot_sync(0xffffffffu, have && mk == tau && rank < need));
-                    if (lane == 0) { sh_lo = tau; sh_hi = tau; sh_need = eq_taken; }
+                    if (lane == 0) { sh.lo = tau; sh.hi = tau; sh.need = eq_taken; }
                 }
                 __syncthreads();
-                lo = sh_lo; hi = sh_hi; need = sh_need;
+                lo = sh.lo; hi = sh.hi; need = sh.need;
                 break;
             }
         }
@@ -338,7 +247,128 @@ score_select_kernel(SelParams p) {
     if (tid == 0) p.sel_count[seq] = static_cast<int32_t>(n_sel);
 }
 
+// Consecutive "chunks" (SCORE_CHUNK blocks of one sequence, sequence-major) are dealt out in
+// equal runs to the CTAs; the grid is sized to what is resident at once (two CTAs per SM), so
+// small workloads get one chunk per CTA and large ones loop.  Warps run through their run
+// without CTA barriers; a barrier and a ticket follow only when the CTA leaves a sequence.
+__global__ void __launch_bounds__(SCORE_THREADS, 2)
+score_select_kernel(SelParams p) {
+    extern __shared__ uint32_t keys[];             // [padded(n_blocks)] in the selecting CTA
+    __shared__ unsigned hist[BINS + BINS / 32 + 1];
+    __shared__ unsigned warp_tot[SCORE_WARPS];
+    __shared__ uint32_t red_lo[SCORE_WARPS], red_hi[SCORE_WARPS];
+    __shared__ uint32_t cand_key[RESOLVE_MAX];
+    __shared__ int cand_idx[RESOLVE_MAX];
+    __shared__ SelShared sh;
+    __shared__ int sh_last;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_chunks = (p.max_blocks + SCORE_CHUNK - 1) / SCORE_CHUNK;
+    const int total = n_chunks * p.batch;
+    const int f1 = min((static_cast<int>(blockIdx.x) + 1) * p.per, total);
+    int f = blockIdx.x * p.per;
+
+    while (f < f1) {
+        const int seq = f / n_chunks;
+        const int fe = min(f1, (seq + 1) * n_chunks);          // this CTA's chunks of this sequence
+        const uint4* dg = p.digest + static_cast<size_t>(seq) * p.max_blocks * 32;   // 32 uint4 per block
+        float w[8];
+        int n_blocks = 0;
+        for (int c = f; c < fe; ++c) {
+            // every load is issued before anything waits: digest rows up to max_blocks are
+            // allocated, so they are read unguarded and masked at the store
+            const int b0 = (c - seq * n_chunks) * SCORE_CHUNK + warp * BLOCKS_PER_WARP;
+            uint4 v[BLOCKS_PER_WARP];
+#pragma unroll
+            for (int i = 0; i < BLOCKS_PER_WARP; ++i) {
+                v[i] = make_uint4(0, 0, 0, 0);
+                if (b0 + i < p.max_blocks) v[i] = ld_stream16(dg + static_cast<size_t>(b0 + i) * 32 + lane);
+            }
+            if (c == f) {
+                // lanes 0-15 hold Q- for channels 8*lane.., lanes 16-31 hold Q+ for channels 8*(lane-16)..
+#pragma unroll
+                for (int i = 0; i < 8; ++i) w[i] = 0.f;
+                const int d0 = (lane & 15) * 8;
+                const bool plus = lane >= 16;
+                const __nv_bfloat16* qh = p.q + (static_cast<size_t>(seq) * p.Hq + static_cast<size_t>(p.h_star) * p.G) * PI_HEAD_DIM + d0;
+                // the group's query rows are fetched four at a time so their latencies overlap
+                for (int g0 = 0; g0 < p.G; g0 += 4) {
+                    uint4 qv[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        qv[j] = make_uint4(0, 0, 0, 0);
+                        if (g0 + j < p.G) qv[j] = *reinterpret_cast<const uint4*>(qh + static_cast<size_t>(g0 + j) * PI_HEAD_DIM);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&qv[j]);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            float2 fv = __bfloat1622float2(h2[i]);
+                            w[2 * i] += plus ? fmaxf(fv.x, 0.f) : fminf(fv.x, 0.f);
+                            w[2 * i + 1] += plus ? fmaxf(fv.y, 0.f) : fminf(fv.y, 0.f);
+                        }
+                    }
+                }
+                int ctx = p.ctx_len[seq];
+                if (ctx < 0) ctx = 0;
+                n_blocks = (ctx + p.B - 1) / p.B;
+                if (n_blocks > p.max_blocks) {
+                    if (tid == 0 && c == seq * n_chunks) pi_report(p.st, PI_ERR_CAPACITY, PI_STAGE_SELECT, seq, n_blocks, p.max_blocks);
+                    n_blocks = p.max_blocks;
+                }
+            }
+            float s[BLOCKS_PER_WARP];
+#pragma unroll
+            for (int i = 0; i < BLOCKS_PER_WARP; ++i) s[i] = dot8(v[i], w);
+            // transposed warp reduction: 8 values x 32 lanes -> lane group (lane>>2) owns block (lane>>2)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const bool up = lane & 16;
+                float send = up ? s[i] : s[i + 4];
+                float keep = up ? s[i + 4] : s[i];
+                s[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+            }
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const bool up = lane & 8;
+                float send = up ? s[i] : s[i + 2];
+                float keep = up ? s[i + 2] : s[i];
+                s[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+            }
+            {
+                const bool up = lane & 4;
+                float send = up ? s[0] : s[1];
+                float keep = up ? s[1] : s[0];
+                s[0] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+            }
+            s[0] += __shfl_xor_sync(0xffffffffu, s[0], 2);
+            s[0] += __shfl_xor_sync(0xffffffffu, s[0], 1);
+            const int b = b0 + (lane >> 2);
+            if ((lane & 3) == 0 && b < n_blocks) p.scores[static_cast<size_t>(seq) * p.max_blocks + b] = s[0];
+        }
+        f = fe;
+
+        // ---------------- ticket: the CTA that completes the sequence selects for it
+        // (the CTA barrier orders every thread's score stores before thread 0's fence and ticket)
+        const int first_cta = (seq * n_chunks) / p.per, last_cta = ((seq + 1) * n_chunks - 1) / p.per;
+        __syncthreads();
+        if (tid == 0) {
+            __threadfence();
+            unsigned t = atomicAdd(&p.counters[seq], 1u);
+            sh_last = (t == static_cast<unsigned>(last_cta - first_cta));
+            if (sh_last) p.counters[seq] = 0;           // ready for the next launch
+            __threadfence();
+        }
+        __syncthreads();
+        if (sh_last) select_sequence(p, seq, n_blocks, keys, hist, warp_tot, red_lo, red_hi, cand_key, cand_idx, sh);
+        __syncthreads();                                // shared arrays are reused by the next sequence
+    }
+}
+
 }  // namespace
+
+static int launch_score_select(SelParams& p, int batch, int n_sms, cudaStream_t stream);
 
 int pi_launch_score_select(pi_ctx* c, int h_star, int batch, const void* q, const void* digest,
                            const int32_t* ctx_len, int32_t* sel, int32_t* sel_count, float* scores,
@@ -360,10 +390,20 @@ int pi_launch_score_select(pi_ctx* c, int h_star, int batch, const void* q, cons
     p.n_sink = c->cfg.n_sink_blocks;
     p.n_local = c->cfg.n_local_blocks;
     p.max_blocks = c->cfg.max_blocks;
-    const size_t smem = (static_cast<size_t>(c->cfg.max_blocks) + c->cfg.max_blocks / 32 + 1) * sizeof(uint32_t);
+    return launch_score_select(p, batch, c->n_sms, stream);
+}
+
+// Grid sizing shared by both entry points: as many CTAs as are resident at once (two per SM),
+// each with an equal run of chunks.
+static int launch_score_select(SelParams& p, int batch, int n_sms, cudaStream_t stream) {
+    const int n_chunks = (p.max_blocks + SCORE_CHUNK - 1) / SCORE_CHUNK;
+    const int total = n_chunks * batch;
+    p.batch = batch;
+    p.per = (total + 2 * n_sms - 1) / (2 * n_sms);
+    const int grid = (total + p.per - 1) / p.per;
+    const size_t smem = (static_cast<size_t>(p.max_blocks) + p.max_blocks / 32 + 1) * sizeof(uint32_t);
     if (smem > 40 * 1024)
         PI_CUDA_TRY(cudaFuncSetAttribute(score_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    dim3 grid((c->cfg.max_blocks + SCORE_CHUNK - 1) / SCORE_CHUNK, batch);
     score_select_kernel<<<grid, SCORE_THREADS, smem, stream>>>(p);
     PI_CUDA_TRY(cudaGetLastError());
     return PI_OK;
@@ -447,9 +487,7 @@ extern "C" int pi_score_select_noalloc(int batch, int n_q_heads, int n_kv_heads,
     p.n_local = n_local_blocks;
     p.max_blocks = max_blocks;
     // at most (8192 + 8192/32 + 1) keys: below the default dynamic shared-memory limit
-    const size_t smem = (static_cast<size_t>(max_blocks) + max_blocks / 32 + 1) * sizeof(uint32_t);
-    dim3 grid((max_blocks + SCORE_CHUNK - 1) / SCORE_CHUNK, batch);
-    score_select_kernel<<<grid, SCORE_THREADS, smem, s>>>(p);
-    PI_CUDA_TRY(cudaGetLastError());
-    return PI_OK;
+    int n_sms = 0;
+    PI_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
+    return launch_score_select(p, batch, n_sms, s);
 }
