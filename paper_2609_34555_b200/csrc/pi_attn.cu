@@ -21,6 +21,7 @@ namespace {
 constexpr int ATTN_MAX_STAGES = 8;
 constexpr int ATTN_META_UNITS = 1024;              // units per CTA whose metadata is staged in shared memory
 constexpr int ATTN_SMEM_BUDGET = 196 * 1024;       // ring bytes
+constexpr int MERGE_BATCH = 12;                    // partial outputs a lane of the merge kernel has in flight
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s: a wait this long is a failure
 
 struct AttnParams {
@@ -156,9 +157,9 @@ attn_merge_kernel(AttnParams p, int main_ctas) {
     const size_t slot0 = static_cast<size_t>(c_first) + seq;
     for (int g = warp; g < p.G; g += n_warps) {
         const size_t head = static_cast<size_t>(h) * p.G + g;
-        // lane i holds (m, l) of segment i (+32, +64, ...).  The first eight partial outputs are
+        // lane i holds (m, l) of segment i (+32, +64, ...).  The first MERGE_BATCH partial outputs are
         // requested in the same breath (they do not depend on the weights), so a sequence cut into
-        // up to eight segments costs one round trip to L2.
+        // up to that many segments costs one round trip to L2.
         float2 ml0 = make_float2(-INFINITY, 0.f);
         float M = -INFINITY;
         for (int sg = lane; sg < n_seg; sg += 32) {
@@ -166,16 +167,16 @@ attn_merge_kernel(AttnParams p, int main_ctas) {
             if (sg < 32) ml0 = ml;
             M = fmaxf(M, ml.x);
         }
-        float4 v[8];
-        auto fetch = [&](int first) {
+        float4 v[MERGE_BATCH];
+        auto fetch = [&](int first, int end) {       // segments [first, first + MERGE_BATCH) below `end`
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
+            for (int kk = 0; kk < MERGE_BATCH; ++kk) {
                 v[kk] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (first + kk < n_seg)
+                if (first + kk < end)
                     v[kk] = __ldcg(reinterpret_cast<const float4*>(p.part_o + ((slot0 + first + kk) * p.Hq + head) * PI_HEAD_DIM) + lane);
             }
         };
-        fetch(0);
+        fetch(0, min(32, n_seg));
 #pragma unroll
         for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -190,10 +191,10 @@ attn_merge_kernel(AttnParams p, int main_ctas) {
                 L += w * ml.y;
             }
             const int cnt = min(32, n_seg - s0);
-            for (int k = 0; k < cnt; k += 8) {
-                if (s0 + k > 0) fetch(s0 + k);
+            for (int k = 0; k < cnt; k += MERGE_BATCH) {
+                if (s0 + k > 0) fetch(s0 + k, s0 + cnt);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
+                for (int kk = 0; kk < MERGE_BATCH; ++kk) {
                     const float wk = __shfl_sync(0xffffffffu, w, (k + kk) & 31);
                     acc.x += wk * v[kk].x; acc.y += wk * v[kk].y; acc.z += wk * v[kk].z; acc.w += wk * v[kk].w;
                 }
