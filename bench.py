@@ -189,13 +189,32 @@ def run_ours(args) -> dict:
             dist.barrier()
         torch.cuda.synchronize()
 
+    # scripted miss counts (config 3): a pre-pass computes every step's selections (they depend
+    # on queries and digests only), then the hot-set contents of every (layer, step) are chosen so
+    # that exactly the drawn heavy-tailed number of selected middle blocks is missing
+    scripts = None
+    if cfg.miss_script == "pareto":
+        from workloads import generate as gen
+        scripts = []
+        b0 = sess.bufs[0]
+        tmp_sel, tmp_cnt = torch.empty_like(b0.sel_blocks), torch.empty_like(b0.sel_count)
+        for tt in range(q_all.shape[0]):
+            per_layer = []
+            for l in range(cfg.n_layers):
+                pi.score_select(l, q_all[tt, l], sess.bufs[l].digest, sess.ctx_len, tmp_sel, tmp_cnt)
+                m = gen.pareto_miss_counts(cfg, l, tt)
+                per_layer.append(gen.scripted_resident_lists(cfg, tmp_sel, tmp_cnt, m, gen.seed_for(cfg, gen.T_PARETO, l, 7919 + tt)))
+            scripts.append(torch.stack(per_layer))
+        torch.cuda.synchronize()
+    script = (lambda i: scripts[i]) if scripts is not None else (lambda i: None)
+
     # settling steps (workload preparation, not warm-up): the hot set starts as a uniform
     # draw, so the first steps recall far more than the steady state does
     t = 0
     for _ in range(args.settle):
-        sess.decode_step(q_all[t]); t += 1
+        sess.decode_step(q_all[t], resident_script=script(t)); t += 1
     for _ in range(W):
-        sess.decode_step(q_all[t]); t += 1
+        sess.decode_step(q_all[t], resident_script=script(t)); t += 1
     barrier()
     pi.stats(reset=True)
 
@@ -207,7 +226,7 @@ def run_ours(args) -> dict:
     barrier()
     e0.record()
     for _ in range(K):
-        sess.decode_step(q_all[t], timer=timer); t += 1
+        sess.decode_step(q_all[t], timer=timer, resident_script=script(t)); t += 1
     e1.record()
     barrier()
     clocks = sampler.stop()
@@ -223,7 +242,7 @@ def run_ours(args) -> dict:
     s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     s0.record()
     for _ in range(n_serial):
-        sess.decode_step(q_all[t], overlapped=False, timer=ser_timer); t += 1
+        sess.decode_step(q_all[t], overlapped=False, timer=ser_timer, resident_script=script(t)); t += 1
     s1.record()
     torch.cuda.synchronize()
     serial_ms = s0.elapsed_time(s1) / max(1, n_serial)
@@ -239,8 +258,9 @@ def run_ours(args) -> dict:
         barrier()
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a0.record()
+        t_e2e = t
         for i in range(n_e2e):
-            sess.decode_step_from_host(q_host[i], out_host, q_dev)
+            sess.decode_step_from_host(q_host[i], out_host, q_dev, resident_script=script(t_e2e + i))
         a1.record()
         barrier()
         e2e_ms = max_over_ranks(a0.elapsed_time(a1), world, dev)
@@ -272,10 +292,12 @@ def run_ours(args) -> dict:
                                f"Hq/Hkv {cfg.n_q_heads}/{cfg.n_kv_heads}, block {cfg.block_tokens}, budget {cfg.budget_blocks} "
                                f"blocks, pool {cfg.pool_slots} slots/seq/layer, AR(1) queries a={cfg.ar1}",
                    "host_kv_layers": R, "host_kv_pinned_gb": R * cfg.batch * cfg.n_blocks * cfg.block_bytes / 2 ** 30,
-                   "l2": "inputs larger than L2 (pool reads 128 MiB and digests 16 MiB per layer-step, all layers distinct)",
+                   "l2": f"inputs larger than L2 (pool reads {cfg.batch * cfg.budget_blocks * cfg.block_bytes / 2**20:.0f} MiB and digests "
+                         f"{cfg.batch * cfg.n_blocks * 512 / 2**20:.0f} MiB per layer-step, {cfg.n_layers} distinct layers)",
                    "pipeline": "select+diff on stream A, recall pulls on stream B, attention on the main stream",
                    "sequence_layer_steps_per_s": world * K * cfg.n_layers * cfg.batch / (ms * 1e-3),
                    "misses_per_seq_layer_step": stats["missing_blocks"] / max(1, stats["sequences"]),
+                   "miss_script": cfg.miss_script or "none (LRU)",
                    "settle_steps": args.settle, "setup_s": round(setup_s, 1)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * n_launch,
         "roofline": {"kernel": "recall_kernel", "bound": "host_link_h2d", "achieved": recall_gbs, "peak": h2d_gbs,

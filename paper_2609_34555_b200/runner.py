@@ -166,9 +166,12 @@ class DecodeSession:
         self._path.prepare_layer(layer, self.bufs[layer], host, self.ctx_len, resident,
                                  kv_for_digest=kv_dev)
 
-    def decode_step(self, q: torch.Tensor, overlapped: bool = True, timer: Optional[StageTimer] = None) -> torch.Tensor:
+    def decode_step(self, q: torch.Tensor, overlapped: bool = True, timer: Optional[StageTimer] = None,
+                    resident_script: Optional[torch.Tensor] = None) -> torch.Tensor:
         """q: device bf16 [n_layers][batch][Hq][D].  Returns self.out ([n_layers][batch][Hq][D]);
-        valid once the current stream has caught up.
+        valid once the current stream has caught up.  resident_script (int32 [n_layers][batch][C]):
+        workloads with scripted miss counts reset each layer's tables to these hot-set contents
+        before the layer's diff (pool contents are not refreshed: timing runs only).
 
         Overlapped form: three streams.  Selection and diff of every layer run ahead on one
         stream, the recall pulls follow on a second one (the host link stays busy back to
@@ -187,6 +190,8 @@ class DecodeSession:
             if overlapped and step > 1:
                 sel_s.wait_event(self._ev_attn[l])         # last step's attention still reads this layer's lists and pool
             tm = timer
+            if resident_script is not None:
+                pi.table_init(resident_script[l], b.block_table, b.slot_block, b.slot_stamp, stream=sel_s)
             t0 = tm.mark(sel_s) if tm and tm.wants("score_select") else None
             pi.score_select(l, q[l], b.digest, self.ctx_len, b.sel_blocks, b.sel_count, b.scores, stream=sel_s)
             t1 = tm.mark(sel_s) if tm and (tm.wants("score_select") or tm.wants("diff")) else None
@@ -215,11 +220,12 @@ class DecodeSession:
                 if t4 is not None: tm.add("attn", t4, t5)
         return self.out
 
-    def decode_step_from_host(self, q_host: torch.Tensor, out_host: torch.Tensor, q_dev: torch.Tensor) -> None:
+    def decode_step_from_host(self, q_host: torch.Tensor, out_host: torch.Tensor, q_dev: torch.Tensor,
+                              resident_script: Optional[torch.Tensor] = None) -> None:
         """End-to-end form: queries come from pinned host memory, results go back to pinned
         host memory; both copies are enqueued on the main stream around the step."""
         q_dev.copy_(q_host, non_blocking=True)
-        self.decode_step(q_dev, overlapped=True)
+        self.decode_step(q_dev, overlapped=True, resident_script=resident_script)
         out_host.copy_(self.out, non_blocking=True)
 
     def miss_blocks(self) -> int:

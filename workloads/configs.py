@@ -28,6 +28,7 @@ class PathConfig:
     steps: int = 1            # decode steps of the scripted run
     overlap: float = 0.0      # target step-to-step selection overlap (0 = independent)
     ar1: float = 0.0          # AR(1) coefficient of the query process giving `overlap`
+    miss_script: str = ""     # "pareto": miss counts per (seq, layer, step) are scripted, not left to LRU
     head_dim: int = 128
     seed: int = 0
 
@@ -84,7 +85,7 @@ CONFIGS = {
                      steps=64, overlap=0.80, ar1=0.93, seed=2),
     # long context, block 32, heavy-tailed scripted miss counts
     "c3": PathConfig("c3", n_layers=32, batch=64, ctx=131072, n_q_heads=32, n_kv_heads=8,
-                     block_tokens=32, budget_blocks=64, resident_frac=0.10, seed=3),
+                     block_tokens=32, budget_blocks=64, resident_frac=0.10, miss_script="pareto", seed=3),
     # 70B-shaped layer stack (G = 8)
     "c4": PathConfig("c4", n_layers=80, batch=8, ctx=65536, n_q_heads=64, n_kv_heads=8,
                      block_tokens=16, budget_blocks=256, resident_frac=0.15,

@@ -147,3 +147,35 @@ def scripted_misses(cfg: PathConfig, total_misses: int, clustered: bool, extra: 
             blocks = np.sort(np.fromiter(chosen, dtype=np.int64))[:m]
         out.append(blocks.astype(np.int32))
     return out
+
+
+def scripted_resident_lists(cfg: PathConfig, sel_blocks: torch.Tensor, sel_count: torch.Tensor,
+                            miss_counts: np.ndarray, seed: int) -> torch.Tensor:
+    """Hot-set contents that make exactly miss_counts[s] of the selected middle blocks of
+    sequence s non-resident: int32 [batch][C] = sink/local blocks, the other selected middle
+    blocks, then unselected filler blocks.  sel_blocks [batch][K] ascending (device or CPU)."""
+    dev = sel_blocks.device
+    batch, K = sel_blocks.shape
+    C, nb = cfg.pool_slots, cfg.n_blocks
+    g = _gen(dev, seed)
+    pin = torch.from_numpy(pinned_blocks(cfg)).to(dev)
+    is_pin = torch.zeros(nb, dtype=torch.bool, device=dev)
+    is_pin[pin.long()] = True
+    valid = torch.arange(K, device=dev)[None, :] < sel_count[:, None]
+    sel = torch.where(valid, sel_blocks, torch.zeros_like(sel_blocks)).long()
+    mid = valid & ~is_pin[sel]                                           # selected middle entries
+    # drop `miss` of the middle entries per sequence: rank random keys among the middle entries
+    keys = torch.rand((batch, K), device=dev, generator=g)
+    keys = torch.where(mid, keys, torch.full_like(keys, 2.0))
+    rank = keys.argsort(dim=1).argsort(dim=1)
+    miss = torch.from_numpy(np.asarray(miss_counts, dtype=np.int64)).to(dev)
+    dropped = mid & (rank < miss[:, None])
+    keep = valid & ~dropped
+    # priority per block: kept selected blocks first, then unselected non-pinned filler, never the dropped ones
+    score = torch.rand((batch, nb), device=dev, generator=g)                # filler in random order
+    rows = torch.arange(batch, device=dev)[:, None].expand(batch, K)
+    score[rows[keep], sel[keep]] = 3.0
+    score[rows[dropped], sel[dropped]] = -1.0
+    score[:, pin.long()] = 4.0
+    order = score.argsort(dim=1, descending=True)[:, :C]
+    return order.to(torch.int32).contiguous()
