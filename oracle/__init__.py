@@ -140,3 +140,14 @@ def layer_step(ctx_len: np.ndarray, max_blocks: int, B: int, Hkv: int, h_star: i
         _p(slot_stamp), _p(pool), _p(r["score"]), _p(r["sel"]), _p(r["sel_count"]),
         _p(r["sel_slots"]), _p(r["miss_pairs"]), _p(r["n_miss"]), _p(r["out"]), _p(r["lse"])))
     return r
+
+
+def append(k_new: np.ndarray, v_new: np.ndarray, ctx: int, B: int, h_star: int, n_sink: int, n_local: int,
+           step: int, host_seq: np.ndarray, pool_seq: np.ndarray, table: np.ndarray, slot_block: np.ndarray,
+           slot_stamp: np.ndarray, digest: np.ndarray) -> int:
+    """Appends one token (k_new, v_new uint16 [Hkv][D]) at position ctx; host store, pool, tables
+    and the digest are updated in place.  Returns the oracle's status code."""
+    Hkv, D = k_new.shape
+    return int(lib().pio_append(_p(np.ascontiguousarray(k_new)), _p(np.ascontiguousarray(v_new)), ctx, B, Hkv, D,
+                                h_star, n_sink, n_local, len(slot_block), ctypes.c_uint32(step), _p(host_seq),
+                                _p(pool_seq), _p(table), _p(slot_block), _p(slot_stamp), _p(digest)))

@@ -292,3 +292,62 @@ int pio_layer_step(int batch, const int32_t* ctx_len, int max_blocks, int B, int
     }
     return rc_all;
 }
+
+/* ---- Append of the step's new token (the step before the recall path; the paper
+ * implies it -- the full KV of an offloaded request lives in CPU memory while sink, local
+ * and hot middle tokens stay on the GPU, Sec. 4.2 / Sec. 5 Setup -- but never describes it:
+ * parity unpinned by the paper, pinned by rebuild-from-scratch invariants in tests/).
+ * The token lands at position p = ctx (length before the append), block b = p / B, row
+ * t = p % B.  A new block (t == 0) belongs to the local window, so it takes a pool slot:
+ * the least recently selected slot whose block is neither sink nor local under the new
+ * length (ties to the lower slot, free slots first); its rows are zeroed in the pool and in
+ * the host store.  The K/V rows of all heads are written to the pool slot and to the host
+ * store, the slot's stamp becomes `step`, and the digest row of block b takes the new key of
+ * the retrieval head into its running min / max.  Returns PIO_OK, or PIO_POOL_TOO_SMALL when
+ * no slot can be evicted, or -8 when a block that must be resident is not. */
+int pio_append(const uint16_t* k_new, const uint16_t* v_new, int ctx, int B, int Hkv, int D, int h_star,
+               int n_sink, int n_local, int C, uint32_t step, uint16_t* host_seq, uint16_t* pool_seq,
+               int32_t* table, int32_t* slot_block, uint32_t* slot_stamp, uint16_t* digest) {
+    int b = ctx / B, t = ctx % B, nb_new = b + 1;
+    size_t blk = (size_t)Hkv * 2 * B * D;
+    int slot = table[b];
+    if (t == 0) {
+        if (slot < 0) {
+            int best = -1;
+            for (int s = 0; s < C; ++s) {
+                int ob = slot_block[s];
+                if (ob >= 0 && is_pinned(ob, nb_new, n_sink, n_local)) continue;
+                if (best < 0 || slot_stamp[s] < slot_stamp[best]) best = s;
+            }
+            if (best < 0) return PIO_POOL_TOO_SMALL;
+            if (slot_block[best] >= 0) table[slot_block[best]] = -1;
+            slot = best;
+            table[b] = slot;
+            slot_block[slot] = b;
+        }
+        memset(pool_seq + (size_t)slot * blk, 0, blk * sizeof(uint16_t));
+        memset(host_seq + (size_t)b * blk, 0, blk * sizeof(uint16_t));
+    } else if (slot < 0) {
+        return -8;
+    }
+    slot_stamp[slot] = step;
+    for (int h = 0; h < Hkv; ++h)
+        for (int d = 0; d < D; ++d) {
+            uint16_t kx = k_new[(size_t)h * D + d], vx = v_new[(size_t)h * D + d];
+            pool_seq[(size_t)slot * blk + in_block(h, 0, t, B, D) + d] = kx;
+            pool_seq[(size_t)slot * blk + in_block(h, 1, t, B, D) + d] = vx;
+            host_seq[(size_t)b * blk + in_block(h, 0, t, B, D) + d] = kx;
+            host_seq[(size_t)b * blk + in_block(h, 1, t, B, D) + d] = vx;
+        }
+    for (int d = 0; d < D; ++d) {
+        uint16_t x = k_new[(size_t)h_star * D + d];
+        uint16_t* lo = digest + ((size_t)b * 2 + 0) * D + d;
+        uint16_t* hi = digest + ((size_t)b * 2 + 1) * D + d;
+        if (t == 0) { *lo = x; *hi = x; }
+        else {
+            if (bf16_val(x) < bf16_val(*lo)) *lo = x;
+            if (bf16_val(x) > bf16_val(*hi)) *hi = x;
+        }
+    }
+    return PIO_OK;
+}
