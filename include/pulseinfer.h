@@ -164,6 +164,27 @@ int pi_sparse_decode_attn(pi_ctx* ctx, int layer, int batch, const void* q_dev, 
                           const int32_t* sel_count_dev, const int32_t* ctx_len_dev, void* out_dev,
                           float* lse_dev, void* stream);
 
+/* The step before the path: the decode step's new token joins the cache.  (The paper implies it:
+ * an offloaded request keeps its full KV in CPU memory and its sink, local and hot middle tokens
+ * on the GPU, Sec. 4.2 and Sec. 5 Setup; it does not describe the operation.)  For every sequence
+ * the token lands at position p = ctx_len[s] (the length BEFORE the append; the caller adds one
+ * afterwards), block b = p / B, row p % B:
+ *   - its K and V rows of all KV heads are written into the pool slot of block b and, through the
+ *     GPU-addressable pinned pointer, into the host store;
+ *   - the digest row of block b takes the retrieval head's new key into its running min / max;
+ *   - a block that has just been opened (p % B == 0) is part of the local window and gets a pool
+ *     slot first: the least recently selected slot whose block is neither sink nor local under
+ *     the new length (ties to the lower slot, free slots first); the evicted block leaves the
+ *     table, the new block's rows start zeroed in the pool and in the host store;
+ *   - the slot's stamp becomes `step`.
+ *   k_new_dev, v_new_dev  [batch][Hkv][D] bf16;  digest_dev [batch][NB][2][D];  other arrays as in
+ *   pi_diff_misses.  Device-side problems (block index beyond NB, nothing evictable, a block that
+ *   must be resident is not) set the status word with stage 5 and leave the sequence untouched. */
+int pi_append_kv(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* k_new_dev,
+                 const void* v_new_dev, const int32_t* ctx_len_dev, void* host_kv_pinned,
+                 int64_t host_seq_stride_bytes, void* pool_dev, int32_t* block_table_dev,
+                 int32_t* slot_block_dev, uint32_t* slot_stamp_dev, void* digest_dev, void* stream);
+
 /* Helpers around the path (input preparation and measurement; not hot calls).
  * pi_build_digests: channel-wise min / max of the keys of head solo_head[layer] over the
  *   valid tokens of each block; kv may be device memory or pinned host memory laid out
@@ -179,7 +200,7 @@ int pi_table_init(pi_ctx* ctx, int batch, const int32_t* resident_dev, int32_t* 
 int pi_h2d_copy_ms(const void* host_pinned, void* dev, int64_t bytes, int reps, float* best_ms);
 
 /* Sticky device status.  out[0] = first PI_ERR_* code seen by a kernel (0 = none),
- * out[1] = stage (1 score/select, 2 diff, 3 recall, 4 attention), out[2..4] = sequence
+ * out[1] = stage (1 score/select, 2 diff, 3 recall, 4 attention, 5 append), out[2..4] = sequence
  * or list, position, offending value.  Reads a pinned mirror: call after the stream
  * has been synchronised.  pi_clear_status resets it. */
 int pi_get_status(pi_ctx* ctx, int32_t out[8]);

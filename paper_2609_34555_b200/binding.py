@@ -23,7 +23,7 @@ ERR_NAMES = {
 EXTENT_DTYPE = torch.int32      # a pi_extent is four int32: src_unit, dst_unit, n_units, units_before
 
 EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_score_select_noalloc", "pi_diff_misses", "pi_recall_gather_scatter",
-           "pi_sparse_decode_attn", "pi_build_digests", "pi_table_init", "pi_h2d_copy_ms",
+           "pi_sparse_decode_attn", "pi_append_kv", "pi_build_digests", "pi_table_init", "pi_h2d_copy_ms",
            "pi_get_status", "pi_get_stats", "pi_clear_status", "pi_strerror"]
 
 
@@ -60,6 +60,7 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.pi_diff_misses.argtypes = [c_void_p, c_int, c_int, c_uint32, i32p, i32p, i32p, i32p, i32p, u32p, i32p, vp, i32p, vp]
     lib.pi_recall_gather_scatter.argtypes = [c_void_p, c_int, c_int, c_int, vp, c_int64, vp, c_int64, vp, c_int32, i32p, c_int64, vp]
     lib.pi_sparse_decode_attn.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, i32p, vp, vp, vp]
+    lib.pi_append_kv.argtypes = [c_void_p, c_int, c_int, c_uint32, vp, vp, i32p, vp, c_int64, vp, i32p, i32p, u32p, vp, vp]
     lib.pi_build_digests.argtypes = [c_void_p, c_int, c_int, vp, c_int64, i32p, vp, vp]
     lib.pi_table_init.argtypes = [c_void_p, c_int, i32p, i32p, i32p, u32p, vp]
     lib.pi_h2d_copy_ms.argtypes = [vp, vp, c_int64, c_int, POINTER(c_float)]
@@ -206,6 +207,20 @@ class PulseInfer:
             _dev(sel_count, torch.int32, "sel_count"), _dev(ctx_len, torch.int32, "ctx_len"),
             _dev(out, torch.bfloat16, "out"), None if lse is None else _dev(lse, torch.float32, "lse"),
             _stream(stream)))
+
+    def append_kv(self, layer: int, step: int, k_new, v_new, ctx_len, host_kv, pool, block_table, slot_block,
+                  slot_stamp, digest, host_seq_stride: Optional[int] = None, stream=None) -> None:
+        """The step's new token (k_new, v_new: [batch][Hkv][D] bf16) joins block ctx_len // B of every
+        sequence: pool slot, host store, running digest; ctx_len is the length before the append."""
+        batch = ctx_len.shape[0]
+        if not host_kv.is_cuda and not host_kv.is_pinned():
+            raise PiError("pi_append_kv", -5, strerror(-5))
+        hs = host_seq_stride if host_seq_stride is not None else host_kv.stride(0) * host_kv.element_size()
+        _check("pi_append_kv", self._lib.pi_append_kv(
+            self._ctx, layer, batch, step, _dev(k_new, torch.bfloat16, "k_new"), _dev(v_new, torch.bfloat16, "v_new"),
+            _dev(ctx_len, torch.int32, "ctx_len"), host_kv.data_ptr(), hs, pool.data_ptr(),
+            _dev(block_table, torch.int32, "block_table"), _dev(slot_block, torch.int32, "slot_block"),
+            _dev(slot_stamp, torch.int32, "slot_stamp"), _dev(digest, torch.bfloat16, "digest"), _stream(stream)))
 
     # ------------------------------------------------------------------ helpers
     def build_digests(self, layer: int, kv, ctx_len, digest, kv_seq_stride: Optional[int] = None, stream=None) -> None:

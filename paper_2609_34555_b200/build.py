@@ -15,7 +15,7 @@ INCLUDE = PKG.parent / "include"
 LIB = PKG / "libpulseinfer_b200.so"
 
 SOURCES = ["pi_api.cu", "pi_score_select.cu", "pi_diff_misses.cu", "pi_recall.cu", "pi_attn.cu",
-           "pi_helpers.cu"]
+           "pi_helpers.cu", "pi_append.cu"]
 
 
 def sources() -> list[Path]:

@@ -181,6 +181,32 @@ extern "C" int pi_sparse_decode_attn(pi_ctx* ctx, int layer, int batch, const vo
                           ctx_len_dev, out_dev, lse_dev, static_cast<cudaStream_t>(stream));
 }
 
+extern "C" int pi_append_kv(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* k_new_dev,
+                            const void* v_new_dev, const int32_t* ctx_len_dev, void* host_kv_pinned,
+                            int64_t host_seq_stride_bytes, void* pool_dev, int32_t* block_table_dev,
+                            int32_t* slot_block_dev, uint32_t* slot_stamp_dev, void* digest_dev, void* stream) {
+    int rc = check_call(ctx, layer, batch);
+    if (rc != PI_OK) return rc;
+    if (!k_new_dev || !v_new_dev || !ctx_len_dev || !host_kv_pinned || !pool_dev || !block_table_dev ||
+        !slot_block_dev || !slot_stamp_dev || !digest_dev || step == 0 || host_seq_stride_bytes < 0)
+        return PI_ERR_INVALID_ARG;
+    if (!pi_aligned16(k_new_dev) || !pi_aligned16(v_new_dev) || !pi_aligned16(host_kv_pinned) ||
+        !pi_aligned16(pool_dev) || !pi_aligned16(digest_dev) || host_seq_stride_bytes % 16)
+        return PI_ERR_BAD_ALIGN;
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, host_kv_pinned) != cudaSuccess) { (void)cudaGetLastError(); return PI_ERR_NOT_PINNED; }
+    void* dst = host_kv_pinned;
+    if (attr.type == cudaMemoryTypeHost) {
+        if (!attr.devicePointer) return PI_ERR_NOT_PINNED;
+        dst = attr.devicePointer;
+    } else if (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged) {
+        return PI_ERR_NOT_PINNED;
+    }
+    return pi_launch_append(ctx, ctx->solo_head[layer], batch, step, k_new_dev, v_new_dev, ctx_len_dev, dst,
+                            host_seq_stride_bytes, pool_dev, block_table_dev, slot_block_dev, slot_stamp_dev,
+                            digest_dev, static_cast<cudaStream_t>(stream));
+}
+
 extern "C" int pi_build_digests(pi_ctx* ctx, int layer, int batch, const void* kv, int64_t kv_seq_stride_bytes,
                                 const int32_t* ctx_len_dev, void* digest_dev, void* stream) {
     int rc = check_call(ctx, layer, batch);

@@ -12,6 +12,7 @@
 #define PI_STAGE_DIFF   2
 #define PI_STAGE_RECALL 3
 #define PI_STAGE_ATTN   4
+#define PI_STAGE_APPEND 5
 
 #define PI_HEAD_DIM 128
 #define PI_SELECT_BINS 2048
@@ -84,6 +85,9 @@ int pi_launch_recall(pi_ctx*, int n_lists, int lists_per_seq, const void* host_k
 int pi_launch_attn(pi_ctx*, int batch, const void* q, const void* pool, const int32_t* sel_slots,
                    const int32_t* sel_blocks, const int32_t* sel_count, const int32_t* ctx_len,
                    void* out, float* lse, cudaStream_t);
+int pi_launch_append(pi_ctx*, int h_star, int batch, uint32_t step, const void* k_new, const void* v_new,
+                     const int32_t* ctx_len, void* host_kv, int64_t host_stride, void* pool, int32_t* table,
+                     int32_t* slot_block, uint32_t* slot_stamp, void* digest, cudaStream_t);
 int pi_launch_build_digests(pi_ctx*, int h_star, int batch, const void* kv, int64_t stride,
                             const int32_t* ctx_len, void* digest, cudaStream_t);
 int pi_launch_table_init(pi_ctx*, int batch, const int32_t* resident, int32_t* table,

@@ -59,10 +59,10 @@ def make_case(cfg, steps: int, ctx_len: Optional[np.ndarray] = None, layer: int 
 
 
 class OracleSide:
-    def __init__(self, case: Case, layer: int = 0):
+    def __init__(self, case: Case, layer: int = 0, own_copy: bool = False):
         cfg = case.cfg
         self.case, self.cfg, self.h = case, cfg, cfg.solo_head(layer)
-        self.kvb = oracle.bits(case.kv)
+        self.kvb = oracle.bits(case.kv).copy() if own_copy else oracle.bits(case.kv)
         nb, C = cfg.n_blocks, cfg.pool_slots
         self.digest = np.zeros((cfg.batch, nb, 2, cfg.head_dim), np.uint16)
         self.table = np.full((cfg.batch, nb), -1, np.int32)
@@ -270,5 +270,79 @@ def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, s
                 assert np.array_equal(b.block_table[s].cpu().numpy(), o["table"])
                 assert np.array_equal(b.slot_stamp[s].cpu().numpy().view(np.uint32), o["slot_stamp"])
                 assert np.array_equal(oracle.bits(b.pool[s].cpu()), o["pool"]), "pool bytes"
+    pi.close()
+    return stats
+
+
+def run_append_and_compare(cfg, steps: int, ctx_len0, layer: int = 0) -> dict:
+    """Decode steps with a growing context: every step first appends one token per sequence
+    (pi_append_kv), then runs the path at the new length.  The oracle keeps its own copy of the
+    host store; at the end both stores, pools, tables and digests must agree bit for bit."""
+    from paper_2609_34555_b200 import PulseInfer
+    from paper_2609_34555_b200.runner import LayerBuffers, RecallPath
+
+    dev = torch.device("cuda:0")
+    case = make_case(cfg, steps, ctx_len=np.asarray(ctx_len0), layer=layer)
+    assert (case.ctx_len + steps <= cfg.n_blocks * cfg.block_tokens).all()
+    g = torch.Generator().manual_seed(gen.seed_for(cfg, 99, layer))
+    new_k = torch.randn((steps, cfg.batch, cfg.n_kv_heads, cfg.head_dim), generator=g).to(torch.bfloat16)
+    new_v = torch.randn((steps, cfg.batch, cfg.n_kv_heads, cfg.head_dim), generator=g).to(torch.bfloat16)
+    pi = PulseInfer.from_workload(cfg)
+    path = RecallPath(pi)
+    buf = LayerBuffers(pi, cfg.batch, dev, keep_scores=True)
+    ctx_d = torch.from_numpy(case.ctx_len.copy()).to(dev)
+    path.prepare_layer(layer, buf, case.kv, ctx_d, torch.from_numpy(case.resident).to(dev))
+    torch.cuda.synchronize()
+    ref = OracleSide(case, layer, own_copy=True)
+    ctx = case.ctx_len.copy()
+    out_d = torch.zeros((cfg.batch, cfg.n_q_heads, cfg.head_dim), dtype=torch.bfloat16, device=dev)
+    stats = dict(max_abs=0.0, new_blocks=0, misses=0)
+    for t in range(steps):
+        step = t + 1
+        kd, vd, q_d = new_k[t].to(dev), new_v[t].to(dev), case.q[t].to(dev)
+        pi.append_kv(layer, step, kd, vd, ctx_d, case.kv, buf.pool, buf.block_table, buf.slot_block, buf.slot_stamp,
+                     buf.digest)
+        ctx_d += 1
+        path.layer_step(layer, step, buf, q_d, ctx_d, case.kv, out_d)
+        torch.cuda.synchronize()
+        assert pi.status()[0] == 0, pi.status()
+        qb, kb, vb = oracle.bits(case.q[t]), oracle.bits(new_k[t]), oracle.bits(new_v[t])
+        g_sel, g_cnt = buf.sel_blocks.cpu().numpy(), buf.sel_count.cpu().numpy()
+        g_slots = buf.sel_slots.cpu().numpy()
+        g_out = out_d.float().cpu().numpy().astype(np.float64)
+        g_dig = oracle.bits(buf.digest.cpu())
+        for s in range(cfg.batch):
+            rc = oracle.append(kb[s], vb[s], int(ctx[s]), cfg.block_tokens, ref.h, cfg.n_sink_blocks, cfg.n_local_blocks,
+                               step, ref.kvb[s], ref.pool[s], ref.table[s], ref.slot_block[s], ref.slot_stamp[s],
+                               ref.digest[s])
+            assert rc == 0
+            stats["new_blocks"] += int(ctx[s] % cfg.block_tokens == 0)
+            ctx[s] += 1
+            n_s = -(-int(ctx[s]) // cfg.block_tokens)
+            assert np.array_equal(g_dig[s, :n_s], ref.digest[s, :n_s]), f"seq {s}: digest after append"
+            sc = oracle.score(qb[s], ref.digest[s], n_s, cfg.n_kv_heads, ref.h)
+            sel_ref, cnt_ref = oracle.select(sc, cfg.n_sink_blocks, cfg.n_local_blocks, cfg.budget_blocks)
+            assert g_cnt[s] == cnt_ref
+            gs, rs = set(g_sel[s, :cnt_ref].tolist()), set(sel_ref[:cnt_ref].tolist())
+            check_near_tie(gs, rs, sc, min(cfg.k_mid, max(0, n_s - cfg.n_sink_blocks - cfg.n_local_blocks)), cfg, n_s)
+            rc, slots, pairs = oracle.diff(g_sel[s], int(g_cnt[s]), n_s, cfg.n_sink_blocks, cfg.n_local_blocks, step,
+                                           ref.table[s], ref.slot_block[s], ref.slot_stamp[s])
+            assert rc == 0 and np.array_equal(g_slots[s], slots)
+            unit = cfg.block_bytes
+            oracle.recall(ref.kvb[s].view(np.uint8).reshape(-1, unit), ref.pool[s].view(np.uint8).reshape(-1, unit), pairs, unit)
+            stats["misses"] += len(pairs)
+            want, _ = oracle.attention(qb[s], ref.pool[s], slots, g_sel[s], int(g_cnt[s]), int(ctx[s]), cfg.block_tokens,
+                                       cfg.n_kv_heads)
+            err = np.abs(g_out[s] - want)
+            stats["max_abs"] = max(stats["max_abs"], float(err.max()))
+            assert np.all(err <= np.maximum(ATTN_MAX_ABS, np.abs(want) * 2.0 ** -8)) and err.mean() <= ATTN_MEAN_ABS
+        assert np.array_equal(buf.block_table.cpu().numpy(), ref.table)
+        assert np.array_equal(buf.slot_block.cpu().numpy(), ref.slot_block)
+        assert np.array_equal(buf.slot_stamp.cpu().numpy().view(np.uint32), ref.slot_stamp)
+        assert np.array_equal(oracle.bits(buf.pool.cpu()), ref.pool), "pool bytes"
+    host = oracle.bits(case.kv)
+    for s in range(cfg.batch):
+        n_s = -(-int(ctx[s]) // cfg.block_tokens)
+        assert np.array_equal(host[s, :n_s], ref.kvb[s, :n_s]), "host store after the appends"
     pi.close()
     return stats

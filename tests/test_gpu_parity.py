@@ -140,3 +140,18 @@ def test_errors_seen_on_the_device_or_at_the_boundary():
     assert all(torch.equal(a, b) for a, b in zip(before, (b2.block_table, b2.slot_block, b2.slot_stamp)))
     pi2.close()
     pi.close()
+
+
+def test_append_then_decode_with_growing_ragged_contexts():
+    from tests.parity import run_append_and_compare
+    cfg = tiny_config(batch=4, ctx=1200, n_q_heads=16, n_kv_heads=4, budget_blocks=24, resident_frac=0.4)
+    # sequences sit at different offsets inside their last block: block boundaries are crossed at different steps
+    stats = run_append_and_compare(cfg, steps=20, ctx_len0=[1000, 1007, 639, 800])
+    assert stats["new_blocks"] >= 4
+
+
+def test_append_block_32_group_of_eight():
+    from tests.parity import run_append_and_compare
+    cfg = tiny_config(batch=2, ctx=2100, n_q_heads=64, n_kv_heads=8, block_tokens=32, budget_blocks=16, resident_frac=0.3)
+    stats = run_append_and_compare(cfg, steps=40, ctx_len0=[2015, 1500])
+    assert stats["new_blocks"] >= 2
