@@ -99,7 +99,7 @@ class ClockSampler:
                     samples=len(sm), reasons=sorted(reasons))
 
 
-def build_session(cfg, rank: int, host_layers_arg: int, world: int, recall_ctas: int = 0):
+def build_session(cfg, rank: int, host_layers_arg: int, world: int, recall_ctas: int = 0, ctx_start: int = 0):
     from paper_2609_34555_b200 import PulseInfer
     from paper_2609_34555_b200.runner import DecodeSession
     from workloads import generate as gen
@@ -112,11 +112,16 @@ def build_session(cfg, rank: int, host_layers_arg: int, world: int, recall_ctas:
         R = int(max(1, min(cfg.n_layers, budget // per_layer)))
     pi = PulseInfer.from_workload(cfg, recall_ctas=recall_ctas)
     sess = DecodeSession(pi, cfg.batch, cfg.n_layers, host_layers=R)
-    sess.ctx_len.fill_(cfg.ctx)
+    ctx0 = ctx_start or cfg.ctx                 # runs that append tokens start short of the full context
+    sess.ctx_len.fill_(ctx0)
     dev = sess.device
+    short = cfg.replace(ctx=ctx0)
     for l in range(cfg.n_layers):
         kv = gen.make_kv(cfg, l, device=dev) if l < R else None
-        res = torch.from_numpy(gen.initial_resident(cfg, l)).to(dev)
+        res_np = np.full((cfg.batch, cfg.pool_slots), -1, np.int32)
+        r0 = gen.initial_resident(short, l)[:, :cfg.pool_slots]
+        res_np[:, :r0.shape[1]] = r0
+        res = torch.from_numpy(res_np).to(dev)
         sess.load_layer(l, kv, res)
         del kv
     torch.cuda.synchronize()
@@ -169,9 +174,11 @@ def run_ours(args) -> dict:
     K, W = args.steps, max(3, args.warmup)
 
     t_setup = time.time()
-    pi, sess, R = build_session(cfg, rank, args.host_layers, world, args.recall_ctas)
     n_e2e = K if not args.no_e2e else 0
     n_serial = min(K, 4)
+    total_steps = args.settle + W + K + n_serial + n_e2e
+    pi, sess, R = build_session(cfg, rank, args.host_layers, world, args.recall_ctas,
+                                ctx_start=cfg.ctx - total_steps - 1 if args.append else 0)
     q_all = make_all_queries(cfg, args.settle + W + K + n_serial + n_e2e, dev)
     setup_s = time.time() - t_setup
 
@@ -207,14 +214,20 @@ def run_ours(args) -> dict:
             scripts.append(torch.stack(per_layer))
         torch.cuda.synchronize()
     script = (lambda i: scripts[i]) if scripts is not None else (lambda i: None)
+    new_kv = None
+    if args.append:
+        gk = torch.Generator(device=dev).manual_seed(cfg.seed * 7 + 1)
+        shape = (cfg.n_layers, cfg.batch, cfg.n_kv_heads, cfg.head_dim)
+        new_kv = (torch.randn(shape, device=dev, generator=gk).to(torch.bfloat16),
+                  torch.randn(shape, device=dev, generator=gk).to(torch.bfloat16))     # the same token values every step
 
     # settling steps (workload preparation, not warm-up): the hot set starts as a uniform
     # draw, so the first steps recall far more than the steady state does
     t = 0
     for _ in range(args.settle):
-        sess.decode_step(q_all[t], resident_script=script(t)); t += 1
+        sess.decode_step(q_all[t], resident_script=script(t), new_kv=new_kv); t += 1
     for _ in range(W):
-        sess.decode_step(q_all[t], resident_script=script(t)); t += 1
+        sess.decode_step(q_all[t], resident_script=script(t), new_kv=new_kv); t += 1
     barrier()
     pi.stats(reset=True)
 
@@ -226,7 +239,7 @@ def run_ours(args) -> dict:
     barrier()
     e0.record()
     for _ in range(K):
-        sess.decode_step(q_all[t], timer=timer, resident_script=script(t)); t += 1
+        sess.decode_step(q_all[t], timer=timer, resident_script=script(t), new_kv=new_kv); t += 1
     e1.record()
     barrier()
     clocks = sampler.stop()
@@ -242,7 +255,7 @@ def run_ours(args) -> dict:
     s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     s0.record()
     for _ in range(n_serial):
-        sess.decode_step(q_all[t], overlapped=False, timer=ser_timer, resident_script=script(t)); t += 1
+        sess.decode_step(q_all[t], overlapped=False, timer=ser_timer, resident_script=script(t), new_kv=new_kv); t += 1
     s1.record()
     torch.cuda.synchronize()
     serial_ms = s0.elapsed_time(s1) / max(1, n_serial)
@@ -297,7 +310,7 @@ def run_ours(args) -> dict:
                    "pipeline": "select+diff on stream A, recall pulls on stream B, attention on the main stream",
                    "sequence_layer_steps_per_s": world * K * cfg.n_layers * cfg.batch / (ms * 1e-3),
                    "misses_per_seq_layer_step": stats["missing_blocks"] / max(1, stats["sequences"]),
-                   "miss_script": cfg.miss_script or "none (LRU)",
+                   "miss_script": cfg.miss_script or "none (LRU)", "append": bool(args.append),
                    "settle_steps": args.settle, "setup_s": round(setup_s, 1)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * n_launch,
         "roofline": {"kernel": "recall_kernel", "bound": "host_link_h2d", "achieved": recall_gbs, "peak": h2d_gbs,
@@ -310,9 +323,9 @@ def run_ours(args) -> dict:
                       hbm_entry("score_select_kernel (pipelined region)", score_bytes_launch, stages["score_select"], traffic.get("score_select_kernel")),
                       hbm_entry("attn_kernel + attn_merge_kernel (serial form, nothing else running)", attn_bytes_launch, ser["attn"], traffic.get("attn_kernel")),
                       hbm_entry("score_select_kernel (serial form)", score_bytes_launch, ser["score_select"], traffic.get("score_select_kernel"))],
-        "stages_us": {k: v["mean_ms"] * 1e3 for k, v in stages.items()},
+        "stages_us": {k: v["mean_ms"] * 1e3 for k, v in stages.items() if v["launches"]},
         "serial": {"layer_steps_per_s": cfg.n_layers / (serial_ms * 1e-3),
-                   "stages_us": {k: v["mean_ms"] * 1e3 for k, v in ser.items()}},
+                   "stages_us": {k: v["mean_ms"] * 1e3 for k, v in ser.items() if v["launches"]}},
         "h2d_peak_gbs": h2d_gbs,
     }
     if rank == 0 and not args.no_cpu and world == 1:
@@ -429,6 +442,7 @@ def main():
     ap.add_argument("--settle", type=int, default=24, help="untimed decode steps before the warm-up")
     ap.add_argument("--layers", type=int, default=0, help="cut the layer stack (for profiler captures only)")
     ap.add_argument("--recall-ctas", type=int, default=0, help="CTAs of the recall kernel (0 = library default)")
+    ap.add_argument("--append", action="store_true", help="grow the context: append one synthetic token per step and layer")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)

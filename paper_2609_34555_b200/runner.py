@@ -96,7 +96,7 @@ class RecallPath:
 class StageTimer:
     """CUDA events around each call of a decode step, on the stream the call runs on."""
 
-    STAGES = ("score_select", "diff", "recall", "attn")
+    STAGES = ("append", "score_select", "diff", "recall", "attn")
 
     def __init__(self, stages=None):
         self.stages = tuple(stages) if stages else self.STAGES
@@ -143,6 +143,7 @@ class DecodeSession:
         self.host_kv = [torch.empty(shape, dtype=torch.bfloat16, pin_memory=True) for _ in range(self.host_layers)]
         self.out = torch.zeros((n_layers, batch, c.n_q_heads, c.head_dim), dtype=torch.bfloat16, device=device)
         self.ctx_len = torch.zeros((batch,), dtype=torch.int32, device=device)
+        self.ctx_prev = torch.zeros((batch,), dtype=torch.int32, device=device)     # length before the step's append
         self.main = torch.cuda.current_stream(self.device)
         self.side = torch.cuda.Stream(self.device)
         self.side2 = torch.cuda.Stream(self.device)
@@ -167,11 +168,13 @@ class DecodeSession:
                                  kv_for_digest=kv_dev)
 
     def decode_step(self, q: torch.Tensor, overlapped: bool = True, timer: Optional[StageTimer] = None,
-                    resident_script: Optional[torch.Tensor] = None) -> torch.Tensor:
+                    resident_script: Optional[torch.Tensor] = None, new_kv=None) -> torch.Tensor:
         """q: device bf16 [n_layers][batch][Hq][D].  Returns self.out ([n_layers][batch][Hq][D]);
         valid once the current stream has caught up.  resident_script (int32 [n_layers][batch][C]):
         workloads with scripted miss counts reset each layer's tables to these hot-set contents
         before the layer's diff (pool contents are not refreshed: timing runs only).
+        new_kv = (k_new, v_new), each bf16 [n_layers][batch][Hkv][D]: the step's new token is appended
+        to every layer first (pool slot, host store, digest) and the context grows by one.
 
         Overlapped form: three streams.  Selection and diff of every layer run ahead on one
         stream, the recall pulls follow on a second one (the host link stays busy back to
@@ -185,6 +188,10 @@ class DecodeSession:
         if overlapped:
             self._ev_start.record(main)
             sel_s.wait_event(self._ev_start)
+        if new_kv is not None:
+            with torch.cuda.stream(sel_s):
+                self.ctx_prev.copy_(self.ctx_len)
+                self.ctx_len += 1
         for l in range(self.n_layers):
             b, host = self.bufs[l], self.host_region(l)
             if overlapped and step > 1:
@@ -192,6 +199,12 @@ class DecodeSession:
             tm = timer
             if resident_script is not None:
                 pi.table_init(resident_script[l], b.block_table, b.slot_block, b.slot_stamp, stream=sel_s)
+            if new_kv is not None:
+                ta = tm.mark(sel_s) if tm and tm.wants("append") else None
+                pi.append_kv(l, step, new_kv[0][l], new_kv[1][l], self.ctx_prev, host, b.pool, b.block_table,
+                             b.slot_block, b.slot_stamp, b.digest, stream=sel_s)
+                if ta is not None:
+                    tm.add("append", ta, tm.mark(sel_s))
             t0 = tm.mark(sel_s) if tm and tm.wants("score_select") else None
             pi.score_select(l, q[l], b.digest, self.ctx_len, b.sel_blocks, b.sel_count, b.scores, stream=sel_s)
             t1 = tm.mark(sel_s) if tm and (tm.wants("score_select") or tm.wants("diff")) else None
