@@ -249,7 +249,8 @@ class CudaNormal:
         self.torch.cuda.synchronize()
 
 
-def run_on_gpu(offload_layers: int = 256, normal_batch: int = 64, normal_ctx: int = 4096, layers: int = 8) -> list:
+def run_on_gpu(offload_layers: int = 256, normal_batch: int = 64, normal_ctx: int = 4096, layers: int = 8,
+               recall_ctas: int = 0) -> list:
     import numpy as np
     import torch
     sys.path.insert(0, str(Path(__file__).resolve().parent.parent))
@@ -259,7 +260,7 @@ def run_on_gpu(offload_layers: int = 256, normal_batch: int = 64, normal_ctx: in
 
     dev = torch.device("cuda:0")
     cfg = get_config("c2").replace(n_layers=layers)
-    pi = PulseInfer.from_workload(cfg)
+    pi = PulseInfer.from_workload(cfg, recall_ctas=recall_ctas)
     sess = DecodeSession(pi, cfg.batch, cfg.n_layers, host_layers=min(4, layers))
     sess.ctx_len.fill_(cfg.ctx)
     for l in range(cfg.n_layers):
@@ -304,6 +305,7 @@ if __name__ == "__main__":
     ap.add_argument("--offload-layers", type=int, default=256)
     ap.add_argument("--normal-batch", type=int, default=64)
     ap.add_argument("--normal-ctx", type=int, default=4096)
+    ap.add_argument("--recall-ctas", type=int, default=0)
     a = ap.parse_args()
-    for r in run_on_gpu(a.offload_layers, a.normal_batch, a.normal_ctx):
+    for r in run_on_gpu(a.offload_layers, a.normal_batch, a.normal_ctx, recall_ctas=a.recall_ctas):
         print(json.dumps(r))

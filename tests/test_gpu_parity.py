@@ -155,3 +155,39 @@ def test_append_block_32_group_of_eight():
     cfg = tiny_config(batch=2, ctx=2100, n_q_heads=64, n_kv_heads=8, block_tokens=32, budget_blocks=16, resident_frac=0.3)
     stats = run_append_and_compare(cfg, steps=40, ctx_len0=[2015, 1500])
     assert stats["new_blocks"] >= 2
+
+
+def test_middle_attention_mass_and_retrieval_head_choice():
+    import oracle
+    import paper_2609_34555_b200 as pkg
+    from paper_2609_34555_b200.mam import choose_solo_head, kv_head_mam, middle_attention_mass
+    from workloads import generate as gen
+    cfg = tiny_config(batch=3, ctx=1500, n_q_heads=16, n_kv_heads=4, budget_blocks=96, resident_frac=1.0)
+    dev = torch.device("cuda:0")
+    kv = gen.make_kv(cfg, 0)
+    # KV heads 0, 1, 3 are made streaming heads (their queries line up with a sink-token key, so
+    # nearly all their attention mass sits outside the middle); head 2 keeps random queries
+    q = gen.make_queries(cfg, 0, 1)[0]
+    G = cfg.group
+    for s in range(cfg.batch):
+        for h in (0, 1, 3):
+            for g in range(h * G, (h + 1) * G):
+                q[s, g] = (kv[s, 0, h, 0, 1].float() * 0.5).to(torch.bfloat16)
+    pi = pkg.PulseInfer.from_workload(cfg)
+    pool = torch.zeros((cfg.batch, cfg.pool_slots) + tuple(kv.shape[2:]), dtype=torch.bfloat16, device=dev)
+    pool[:, :cfg.n_blocks] = kv.to(dev)
+    ctx = torch.tensor([1500, 1111, 700], dtype=torch.int32, device=dev)
+    mam = middle_attention_mass(pi, 0, q.to(dev), pool, ctx).cpu().numpy()
+    kvb, qb = oracle.bits(kv), oracle.bits(q)
+    for s in range(cfg.batch):
+        nb = -(-int(ctx[s]) // cfg.block_tokens)
+        allb = np.arange(nb, dtype=np.int32)
+        mid = np.arange(cfg.n_sink_blocks, nb - cfg.n_local_blocks, dtype=np.int32)
+        _, la = oracle.attention(qb[s], kvb[s], allb, allb, nb, int(ctx[s]), cfg.block_tokens, cfg.n_kv_heads)
+        _, lm = oracle.attention(qb[s], kvb[s], mid, mid, len(mid), int(ctx[s]), cfg.block_tokens, cfg.n_kv_heads)
+        np.testing.assert_allclose(mam[s], np.exp(lm - la), rtol=2e-3, atol=1e-4)
+    assert choose_solo_head(torch.from_numpy(mam), cfg.n_kv_heads) == 2
+    assert choose_solo_head(torch.from_numpy(mam), cfg.n_kv_heads, reversed_rank=True) != 2
+    assert kv_head_mam(torch.from_numpy(mam), cfg.n_kv_heads).shape == (4,)
+    assert pi.status()[0] == 0
+    pi.close()

@@ -393,3 +393,20 @@ def test_layer_step_is_the_composition_of_its_stages():
             for j in range(cnt):
                 assert np.array_equal(pool[s, slots[j]], kvb[s, sel[j]])
         assert np.array_equal(pool, pool2) and np.array_equal(table, t2)
+
+
+# ----------------------------------------------------------------- Middle Attention Mass (Eq. 2)
+def test_attention_mass_of_a_token_set_from_two_logsumexps():
+    """sum_{i in S} A(i) = exp(lse_S - lse_all): the identity the MAM helper relies on, checked
+    against the softmax weights written out."""
+    ctx, B, Hq, Hkv = 400, 16, 8, 2
+    _, nb, kv, q = _case(31, ctx, B, Hq, Hkv)
+    allb = np.arange(nb, dtype=np.int32)
+    mid = np.arange(1, nb - 8, dtype=np.int32)
+    _, lse_all = oracle.attention(q, kv, allb, allb, nb, ctx, B, Hkv)
+    _, lse_mid = oracle.attention(q, kv, mid, mid, len(mid), ctx, B, Hkv)
+    qf, kf = oracle.bf16_to_f64(q), oracle.bf16_to_f64(kv)[:, :, 0]
+    for g in range(Hq):
+        s = (kf[:, g // (Hq // Hkv)].reshape(-1, 128)[:ctx] @ qf[g]) / np.sqrt(128.0)
+        w = np.exp(s - s.max()); w /= w.sum()
+        np.testing.assert_allclose(np.exp(lse_mid[g] - lse_all[g]), w[B:(nb - 8) * B].sum(), rtol=1e-10)
