@@ -111,7 +111,15 @@ def build_session(cfg, rank: int, host_layers_arg: int, world: int, recall_ctas:
         budget = 0.55 * mem_available_bytes() / max(1, world)
         R = int(max(1, min(cfg.n_layers, budget // per_layer)))
     pi = PulseInfer.from_workload(cfg, recall_ctas=recall_ctas)
-    sess = DecodeSession(pi, cfg.batch, cfg.n_layers, host_layers=R)
+    while True:                                  # pinning can fail below the MemAvailable estimate: halve and retry
+        try:
+            sess = DecodeSession(pi, cfg.batch, cfg.n_layers, host_layers=R)
+            break
+        except RuntimeError:
+            if R == 1:
+                raise
+            R = max(1, R // 2)
+            torch.cuda.empty_cache()
     ctx0 = ctx_start or cfg.ctx                 # runs that append tokens start short of the full context
     sess.ctx_len.fill_(ctx0)
     dev = sess.device
