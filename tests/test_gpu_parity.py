@@ -191,3 +191,63 @@ def test_middle_attention_mass_and_retrieval_head_choice():
     assert kv_head_mam(torch.from_numpy(mam), cfg.n_kv_heads).shape == (4,)
     assert pi.status()[0] == 0
     pi.close()
+
+
+def _carve(total_bytes_list, dev, pattern=0x5A):
+    """One allocation holding every buffer with 4 KB guard zones before, between and after."""
+    guard = 4096
+    offs, pos = [], guard
+    for n in total_bytes_list:
+        pos = (pos + 255) // 256 * 256
+        offs.append(pos)
+        pos += n + guard
+    arena = torch.full((pos + guard,), pattern, dtype=torch.uint8, device=dev)
+    return arena, offs
+
+
+def test_guard_zones_stay_intact_and_results_repeat_bit_for_bit():
+    """No out-of-bounds write anywhere on the path (guard zones around every buffer the kernels
+    write), and two runs from the same state give identical bytes everywhere."""
+    import paper_2609_34555_b200 as pkg
+    from workloads import generate as gen
+    cfg = tiny_config(batch=3, ctx=3000, n_q_heads=32, n_kv_heads=8, budget_blocks=40, resident_frac=0.3)
+    dev = torch.device("cuda:0")
+    pi = pkg.PulseInfer.from_workload(cfg)
+    nb, C, K, Hq = cfg.n_blocks, cfg.pool_slots, cfg.budget_blocks, cfg.n_q_heads
+    shapes = dict(digest=((cfg.batch, nb, 2, 128), torch.bfloat16), table=((cfg.batch, nb), torch.int32),
+                  slot_block=((cfg.batch, C), torch.int32), slot_stamp=((cfg.batch, C), torch.int32),
+                  pool=((cfg.batch, C, 8, 2, 16, 128), torch.bfloat16), sel=((cfg.batch, K), torch.int32),
+                  cnt=((cfg.batch,), torch.int32), slots=((cfg.batch, K), torch.int32),
+                  lst=((cfg.batch, K, 4), torch.int32), lcnt=((cfg.batch,), torch.int32),
+                  out=((cfg.batch, Hq, 128), torch.bfloat16), lse=((cfg.batch, Hq), torch.float32),
+                  scores=((cfg.batch, nb), torch.float32))
+    sizes = [int(np.prod(s)) * torch.empty((), dtype=d).element_size() for s, d in shapes.values()]
+    kv = gen.make_kv(cfg, 0).pin_memory()
+    q = gen.make_queries(cfg, 0, 3, ar1=0.8).to(dev)
+    ctx = torch.tensor([3000, 2990, 1600], dtype=torch.int32, device=dev)
+    res = torch.from_numpy(gen.initial_resident(cfg.replace(ctx=1600), 0)[:, :C]).to(dev)   # valid for the shortest sequence
+    res = torch.nn.functional.pad(res, (0, C - res.shape[1]), value=-1).contiguous()
+    results = []
+    for run in range(2):
+        arena, offs = _carve(sizes, dev)
+        t = {}
+        for (name, (shape, dt)), off, n in zip(shapes.items(), offs, sizes):
+            t[name] = arena[off:off + n].view(dt).view(shape)
+        covered = torch.zeros(arena.numel(), dtype=torch.bool, device=dev)
+        for off, n in zip(offs, sizes):
+            covered[off:off + n] = True
+        t["pool"].zero_()
+        pi.build_digests(0, kv, ctx, t["digest"])
+        pi.table_init(res, t["table"], t["slot_block"], t["slot_stamp"])
+        for step in range(1, 4):
+            pi.score_select(0, q[step - 1], t["digest"], ctx, t["sel"], t["cnt"], t["scores"])
+            pi.diff_misses(0, step, ctx, t["sel"], t["cnt"], t["table"], t["slot_block"], t["slot_stamp"], t["slots"],
+                           t["lst"], t["lcnt"])
+            pi.recall_gather_scatter(0, kv, t["pool"], t["lst"], t["lcnt"])
+            pi.sparse_decode_attn(0, q[step - 1], t["pool"], t["slots"], t["sel"], t["cnt"], ctx, t["out"], t["lse"])
+        torch.cuda.synchronize()
+        assert pi.status()[0] == 0
+        assert bool((arena[~covered] == 0x5A).all()), "a guard zone was written"
+        results.append(arena.clone())
+    assert torch.equal(results[0], results[1]), "two identical runs differ"
+    pi.close()
