@@ -251,3 +251,20 @@ def test_guard_zones_stay_intact_and_results_repeat_bit_for_bit():
         results.append(arena.clone())
     assert torch.equal(results[0], results[1]), "two identical runs differ"
     pi.close()
+
+
+def test_empty_sequence_in_the_batch():
+    from tests.parity import make_case, run_and_compare
+    cfg = tiny_config(batch=3, ctx=1000)
+    case = make_case(cfg, steps=3, ctx_len=np.asarray([1000, 0, 7]))     # nothing, and less than one block
+    run_and_compare(case, steps=3)
+
+
+def test_largest_supported_block_count_and_wide_budget():
+    """16384 blocks per sequence (the library's limit), 512-block budget, 1024-slot pool."""
+    from tests.parity import make_case, run_and_compare
+    cfg = tiny_config(batch=1, ctx=262144, n_q_heads=8, n_kv_heads=2, budget_blocks=512, resident_frac=1024 / 16384)
+    assert cfg.n_blocks == 16384 and cfg.pool_slots == 1024
+    case = make_case(cfg, steps=2)
+    stats = run_and_compare(case, steps=2)
+    assert stats["misses"][0] > 100
