@@ -151,3 +151,27 @@ def append(k_new: np.ndarray, v_new: np.ndarray, ctx: int, B: int, h_star: int, 
     return int(lib().pio_append(_p(np.ascontiguousarray(k_new)), _p(np.ascontiguousarray(v_new)), ctx, B, Hkv, D,
                                 h_star, n_sink, n_local, len(slot_block), ctypes.c_uint32(step), _p(host_seq),
                                 _p(pool_seq), _p(table), _p(slot_block), _p(slot_stamp), _p(digest)))
+
+
+def build_digest_all(kv_seq: np.ndarray, ctx: int) -> np.ndarray:
+    """kv_seq uint16 [n_blocks][Hkv][2][B][D] -> digests of every KV head, uint16 [n_blocks][Hkv][2][D]."""
+    nb, Hkv, _, B, D = kv_seq.shape
+    out = np.zeros((nb, Hkv, 2, D), dtype=np.uint16)
+    lib().pio_build_digest_all(_p(kv_seq), ctx, B, Hkv, D, _p(out))
+    return out
+
+
+def score_heads(q: np.ndarray, digest_all: np.ndarray, n_blocks: int, h_lo: int, h_hi: int) -> np.ndarray:
+    """Sum of the per-head query-digest scores of KV heads [h_lo, h_hi)."""
+    Hq, D = q.shape
+    Hkv = digest_all.shape[1]
+    out = np.zeros(n_blocks, dtype=np.float64)
+    lib().pio_score_heads(_p(q), _p(digest_all), n_blocks, Hq, Hkv, D, h_lo, h_hi, _p(out))
+    return out
+
+
+def recall_strided(host_seq: np.ndarray, pool_seq: np.ndarray, pairs: np.ndarray, unit_bytes: int,
+                   unit_stride: int, offset: int) -> None:
+    pairs = np.ascontiguousarray(pairs, dtype=np.int32)
+    lib().pio_recall_strided(_p(host_seq), _p(pool_seq), _p(pairs), len(pairs), ctypes.c_int64(unit_bytes),
+                             ctypes.c_int64(unit_stride), ctypes.c_int64(offset))

@@ -351,3 +351,53 @@ int pio_append(const uint16_t* k_new, const uint16_t* v_new, int ctx, int B, int
     }
     return PIO_OK;
 }
+
+/* ---- The comparison strategies of Sec. 4.4.1 (headwise: every KV head selects for itself;
+ * average: the per-head query-digest scores are combined and one top-k is shared).  They need
+ * the digests of all KV heads: digest_all[n_blocks][Hkv][2][D].  The score of a set of KV heads
+ * [h_lo, h_hi) is the sum of their per-head scores (a sum ranks like the paper's average):
+ * headwise uses one head at a time, average uses all of them. */
+void pio_build_digest_all(const uint16_t* kv_seq, int ctx, int B, int Hkv, int D, uint16_t* digest_all) {
+    int n_blocks = (ctx + B - 1) / B;
+    size_t blk = (size_t)Hkv * 2 * B * D;
+    for (int b = 0; b < n_blocks; ++b) {
+        int valid = ctx - b * B < B ? ctx - b * B : B;
+        for (int h = 0; h < Hkv; ++h)
+            for (int d = 0; d < D; ++d) {
+                uint16_t lo = kv_seq[b * blk + in_block(h, 0, 0, B, D) + d], hi = lo;
+                for (int t = 1; t < valid; ++t) {
+                    uint16_t x = kv_seq[b * blk + in_block(h, 0, t, B, D) + d];
+                    if (bf16_val(x) < bf16_val(lo)) lo = x;
+                    if (bf16_val(x) > bf16_val(hi)) hi = x;
+                }
+                digest_all[(((size_t)b * Hkv + h) * 2 + 0) * D + d] = lo;
+                digest_all[(((size_t)b * Hkv + h) * 2 + 1) * D + d] = hi;
+            }
+    }
+}
+
+void pio_score_heads(const uint16_t* q, const uint16_t* digest_all, int n_blocks, int Hq, int Hkv, int D,
+                     int h_lo, int h_hi, double* score) {
+    int G = Hq / Hkv;
+    for (int b = 0; b < n_blocks; ++b) {
+        double s = 0.0;
+        for (int h = h_lo; h < h_hi; ++h)
+            for (int g = h * G; g < (h + 1) * G; ++g)
+                for (int d = 0; d < D; ++d) {
+                    double qv = bf16_val(q[(size_t)g * D + d]);
+                    double a = qv * bf16_val(digest_all[(((size_t)b * Hkv + h) * 2 + 0) * D + d]);
+                    double c = qv * bf16_val(digest_all[(((size_t)b * Hkv + h) * 2 + 1) * D + d]);
+                    s += a > c ? a : c;
+                }
+        score[b] = s;
+    }
+}
+
+/* Recall of units that are `unit_bytes` long but `unit_stride` apart, starting `offset` bytes into
+ * the sequence's region: the per-head form of Sec. 3.4 (one (block, head) fragment per transfer). */
+void pio_recall_strided(const uint8_t* host_seq, uint8_t* pool_seq, const int32_t* pairs, int n,
+                        int64_t unit_bytes, int64_t unit_stride, int64_t offset) {
+    for (int i = 0; i < n; ++i)
+        memcpy(pool_seq + offset + (size_t)pairs[2 * i + 1] * unit_stride,
+               host_seq + offset + (size_t)pairs[2 * i] * unit_stride, (size_t)unit_bytes);
+}
