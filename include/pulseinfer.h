@@ -117,6 +117,26 @@ int pi_score_select_noalloc(int batch, int n_q_heads, int n_kv_heads, int block_
                             const int32_t* ctx_len_dev, int32_t* sel_blocks_dev, int32_t* sel_count_dev,
                             int32_t* status_dev, void* stream);
 
+/* The two comparison strategies of the paper's selection study (Sec. 4.4.1), for the
+ * fragmentation story end to end.  Both read digests of EVERY KV head,
+ *   digest_all_dev [batch][NB][Hkv][2][D] bf16 (pi_build_digests_all),
+ * and score a KV head with the queries of its own group.
+ *   PI_SELECT_AVERAGE   the per-head scores are summed (a sum ranks like the paper's average) and
+ *                       one top-k is shared by all heads: sel_blocks_dev [batch][K], sel_count_dev [batch]
+ *   PI_SELECT_HEADWISE  every KV head selects for itself: sel_blocks_dev [batch][Hkv][K],
+ *                       sel_count_dev [batch][Hkv]; needs max_batch >= batch*Hkv
+ * scores_dev: NULL or float [rows][NB], rows = batch or batch*Hkv.  Everything else as pi_score_select.
+ * Per-head selections go through pi_diff_misses with batch*Hkv rows (tables, slot arrays and a
+ * ctx_len array of that many rows) and through pi_recall_gather_scatter with lists_per_seq = Hkv,
+ * unit_bytes = frag_bytes, unit_stride_bytes = block_bytes, list_offset_bytes = frag_bytes: head h
+ * of slot s then holds the fragment of whatever block head h selected.  Attention over per-head
+ * selections is not provided. */
+#define PI_SELECT_AVERAGE  1
+#define PI_SELECT_HEADWISE 2
+int pi_score_select_strategy(pi_ctx* ctx, int strategy, int layer, int batch, const void* q_dev,
+                             const void* digest_all_dev, const int32_t* ctx_len_dev,
+                             int32_t* sel_blocks_dev, int32_t* sel_count_dev, float* scores_dev, void* stream);
+
 /* Step 2 of the workflow (Sec. 2.2): B_recall = B_topk \ B_gpu against the
  * device-resident block table, victim choice (least recently selected slot, ties to
  * the lower slot; sink / local / selected blocks are never evicted), table update,
@@ -145,12 +165,16 @@ int pi_diff_misses(pi_ctx* ctx, int layer, int batch, uint32_t step, const int32
  *   host_kv_pinned           sequence s starts at host_kv_pinned + s*host_seq_stride_bytes
  *   pool_dev                 sequence s starts at pool_dev + s*pool_seq_stride_bytes
  *   recall_list_dev          [n_lists][list_capacity] pi_extent; recall_count_dev [n_lists]
- *   unit_bytes               multiple of 4096 */
+ *   unit_bytes               multiple of 4096
+ *   unit_stride_bytes        distance between consecutive units (0 = unit_bytes: units are contiguous)
+ *   list_offset_bytes        list i starts (i % lists_per_seq) * list_offset_bytes into its sequence's
+ *                            region, in the host store and in the pool alike (0 for the shared selection) */
 int pi_recall_gather_scatter(pi_ctx* ctx, int layer, int n_lists, int lists_per_seq,
                              const void* host_kv_pinned, int64_t host_seq_stride_bytes,
                              void* pool_dev, int64_t pool_seq_stride_bytes,
                              const pi_extent* recall_list_dev, int32_t list_capacity,
-                             const int32_t* recall_count_dev, int64_t unit_bytes, void* stream);
+                             const int32_t* recall_count_dev, int64_t unit_bytes, int64_t unit_stride_bytes,
+                             int64_t list_offset_bytes, void* stream);
 
 /* Attention of the layer over the selected blocks only (Sec. 4.2.1: after the recall
  * completes the offload batch attends over the recalled blocks): for every query
@@ -195,6 +219,9 @@ int pi_append_kv(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* k
  *   host to device memory (the link's reference bandwidth). Synchronises. */
 int pi_build_digests(pi_ctx* ctx, int layer, int batch, const void* kv, int64_t kv_seq_stride_bytes,
                      const int32_t* ctx_len_dev, void* digest_dev, void* stream);
+/* the same for every KV head: digest_all_dev [batch][NB][Hkv][2][D] */
+int pi_build_digests_all(pi_ctx* ctx, int batch, const void* kv, int64_t kv_seq_stride_bytes,
+                         const int32_t* ctx_len_dev, void* digest_all_dev, void* stream);
 int pi_table_init(pi_ctx* ctx, int batch, const int32_t* resident_dev, int32_t* block_table_dev,
                   int32_t* slot_block_dev, uint32_t* slot_stamp_dev, void* stream);
 int pi_h2d_copy_ms(const void* host_pinned, void* dev, int64_t bytes, int reps, float* best_ms);

@@ -22,8 +22,8 @@ ERR_NAMES = {
 }
 EXTENT_DTYPE = torch.int32      # a pi_extent is four int32: src_unit, dst_unit, n_units, units_before
 
-EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_score_select_noalloc", "pi_diff_misses", "pi_recall_gather_scatter",
-           "pi_sparse_decode_attn", "pi_append_kv", "pi_build_digests", "pi_table_init", "pi_h2d_copy_ms",
+EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_score_select_noalloc", "pi_score_select_strategy", "pi_diff_misses", "pi_recall_gather_scatter",
+           "pi_sparse_decode_attn", "pi_append_kv", "pi_build_digests", "pi_build_digests_all", "pi_table_init", "pi_h2d_copy_ms",
            "pi_get_status", "pi_get_stats", "pi_clear_status", "pi_strerror"]
 
 
@@ -58,7 +58,10 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.pi_score_select.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, vp, vp]
     lib.pi_score_select_noalloc.argtypes = [c_int] * 9 + [vp, vp, i32p, i32p, i32p, i32p, vp]
     lib.pi_diff_misses.argtypes = [c_void_p, c_int, c_int, c_uint32, i32p, i32p, i32p, i32p, i32p, u32p, i32p, vp, i32p, vp]
-    lib.pi_recall_gather_scatter.argtypes = [c_void_p, c_int, c_int, c_int, vp, c_int64, vp, c_int64, vp, c_int32, i32p, c_int64, vp]
+    lib.pi_recall_gather_scatter.argtypes = [c_void_p, c_int, c_int, c_int, vp, c_int64, vp, c_int64, vp, c_int32, i32p,
+                                             c_int64, c_int64, c_int64, vp]
+    lib.pi_score_select_strategy.argtypes = [c_void_p, c_int, c_int, c_int, vp, vp, i32p, i32p, i32p, vp, vp]
+    lib.pi_build_digests_all.argtypes = [c_void_p, c_int, vp, c_int64, i32p, vp, vp]
     lib.pi_sparse_decode_attn.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, i32p, vp, vp, vp]
     lib.pi_append_kv.argtypes = [c_void_p, c_int, c_int, c_uint32, vp, vp, i32p, vp, c_int64, vp, i32p, i32p, u32p, vp, vp]
     lib.pi_build_digests.argtypes = [c_void_p, c_int, c_int, vp, c_int64, i32p, vp, vp]
@@ -170,6 +173,25 @@ class PulseInfer:
             _dev(sel_count, torch.int32, "sel_count"),
             None if scores is None else _dev(scores, torch.float32, "scores"), _stream(stream)))
 
+    AVERAGE, HEADWISE = 1, 2
+
+    def score_select_strategy(self, strategy: int, layer: int, q, digest_all, ctx_len, sel_blocks, sel_count,
+                              scores=None, stream=None) -> None:
+        """Averaged (shared) or headwise (per KV head) selection over digests of every KV head."""
+        batch = q.shape[0]
+        _check("pi_score_select_strategy", self._lib.pi_score_select_strategy(
+            self._ctx, strategy, layer, batch, _dev(q, torch.bfloat16, "q"), _dev(digest_all, torch.bfloat16, "digest_all"),
+            _dev(ctx_len, torch.int32, "ctx_len"), _dev(sel_blocks, torch.int32, "sel_blocks"),
+            _dev(sel_count, torch.int32, "sel_count"),
+            None if scores is None else _dev(scores, torch.float32, "scores"), _stream(stream)))
+
+    def build_digests_all(self, kv, ctx_len, digest_all, kv_seq_stride: Optional[int] = None, stream=None) -> None:
+        batch = ctx_len.shape[0]
+        stride = kv_seq_stride if kv_seq_stride is not None else kv.stride(0) * kv.element_size()
+        _check("pi_build_digests_all", self._lib.pi_build_digests_all(
+            self._ctx, batch, kv.data_ptr(), stride, _dev(ctx_len, torch.int32, "ctx_len"),
+            _dev(digest_all, torch.bfloat16, "digest_all"), _stream(stream)))
+
     def diff_misses(self, layer: int, step: int, ctx_len, sel_blocks, sel_count, block_table, slot_block, slot_stamp,
                     sel_slots, recall_list, recall_count, stream=None) -> None:
         batch = sel_count.shape[0]
@@ -183,7 +205,8 @@ class PulseInfer:
 
     def recall_gather_scatter(self, layer: int, host_kv, pool, recall_list, recall_count, *, lists_per_seq: int = 1,
                               unit_bytes: Optional[int] = None, host_seq_stride: Optional[int] = None,
-                              pool_seq_stride: Optional[int] = None, stream=None) -> None:
+                              pool_seq_stride: Optional[int] = None, unit_stride: int = 0, list_offset: int = 0,
+                              stream=None) -> None:
         """host_kv: pinned host tensor [batch][NB] blocks; pool: CUDA tensor [batch][C] blocks;
         recall_list: int32 [n_lists][capacity][4]."""
         n_lists, cap = recall_list.shape[0], recall_list.shape[1]
@@ -194,7 +217,7 @@ class PulseInfer:
         _check("pi_recall_gather_scatter", self._lib.pi_recall_gather_scatter(
             self._ctx, layer, n_lists, lists_per_seq, host_kv.data_ptr(), hs, pool.data_ptr(), ps,
             _dev(recall_list, EXTENT_DTYPE, "recall_list"), cap, _dev(recall_count, torch.int32, "recall_count"),
-            unit_bytes or self.block_bytes, _stream(stream)))
+            unit_bytes or self.block_bytes, unit_stride, list_offset, _stream(stream)))
 
     def sparse_decode_attn(self, layer: int, q, pool, sel_slots, sel_blocks, sel_count, ctx_len, out, lse=None,
                            stream=None) -> None:

@@ -121,6 +121,22 @@ extern "C" int pi_score_select(pi_ctx* ctx, int layer, int batch, const void* q_
                                   ctx->sel_counters, static_cast<cudaStream_t>(stream));
 }
 
+extern "C" int pi_score_select_strategy(pi_ctx* ctx, int strategy, int layer, int batch, const void* q_dev,
+                                       const void* digest_all_dev, const int32_t* ctx_len_dev,
+                                       int32_t* sel_blocks_dev, int32_t* sel_count_dev, float* scores_dev,
+                                       void* stream) {
+    int rc = check_call(ctx, layer, batch);
+    if (rc != PI_OK) return rc;
+    if (strategy != PI_SELECT_AVERAGE && strategy != PI_SELECT_HEADWISE) return PI_ERR_INVALID_ARG;
+    if (!q_dev || !digest_all_dev || !ctx_len_dev || !sel_blocks_dev || !sel_count_dev) return PI_ERR_INVALID_ARG;
+    if (!pi_aligned16(q_dev) || !pi_aligned16(digest_all_dev)) return PI_ERR_BAD_ALIGN;
+    const int n_virtual = strategy == PI_SELECT_HEADWISE ? batch * ctx->cfg.n_kv_heads : batch;
+    if (n_virtual > ctx->cfg.max_batch) return PI_ERR_CAPACITY;      // scratch holds max_batch score rows
+    return pi_launch_score_select_strategy(ctx, strategy, batch, q_dev, digest_all_dev, ctx_len_dev, sel_blocks_dev,
+                                           sel_count_dev, scores_dev ? scores_dev : ctx->scores, ctx->sel_counters,
+                                           static_cast<cudaStream_t>(stream));
+}
+
 extern "C" int pi_diff_misses(pi_ctx* ctx, int layer, int batch, uint32_t step, const int32_t* ctx_len_dev,
                               const int32_t* sel_blocks_dev, const int32_t* sel_count_dev,
                               int32_t* block_table_dev, int32_t* slot_block_dev, uint32_t* slot_stamp_dev,
@@ -141,12 +157,16 @@ extern "C" int pi_recall_gather_scatter(pi_ctx* ctx, int layer, int n_lists, int
                                         const void* host_kv_pinned, int64_t host_seq_stride_bytes,
                                         void* pool_dev, int64_t pool_seq_stride_bytes,
                                         const pi_extent* recall_list_dev, int32_t list_capacity,
-                                        const int32_t* recall_count_dev, int64_t unit_bytes, void* stream) {
+                                        const int32_t* recall_count_dev, int64_t unit_bytes,
+                                        int64_t unit_stride_bytes, int64_t list_offset_bytes, void* stream) {
     if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers) return PI_ERR_INVALID_ARG;
     if (n_lists < 1 || lists_per_seq < 1 || n_lists % lists_per_seq || n_lists > 65536) return PI_ERR_INVALID_ARG;
     if (!host_kv_pinned || !pool_dev || !recall_list_dev || !recall_count_dev || list_capacity < 1)
         return PI_ERR_INVALID_ARG;
     if (unit_bytes < 4096 || unit_bytes % 4096 || unit_bytes > (1 << 24)) return PI_ERR_UNSUPPORTED_DIM;
+    if (unit_stride_bytes < 0 || (unit_stride_bytes > 0 && unit_stride_bytes < unit_bytes) || unit_stride_bytes % 16 ||
+        list_offset_bytes < 0 || list_offset_bytes % 16)
+        return PI_ERR_INVALID_ARG;
     if (host_seq_stride_bytes % 16 || pool_seq_stride_bytes % 16 || host_seq_stride_bytes < 0 ||
         pool_seq_stride_bytes < 0)
         return PI_ERR_BAD_ALIGN;
@@ -164,7 +184,7 @@ extern "C" int pi_recall_gather_scatter(pi_ctx* ctx, int layer, int n_lists, int
     }
     return pi_launch_recall(ctx, n_lists, lists_per_seq, src, host_seq_stride_bytes, pool_dev,
                             pool_seq_stride_bytes, recall_list_dev, list_capacity, recall_count_dev,
-                            unit_bytes, static_cast<cudaStream_t>(stream));
+                            unit_bytes, unit_stride_bytes, list_offset_bytes, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int pi_sparse_decode_attn(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* pool_dev,
@@ -224,6 +244,25 @@ extern "C" int pi_build_digests(pi_ctx* ctx, int layer, int batch, const void* k
     }
     return pi_launch_build_digests(ctx, ctx->solo_head[layer], batch, src, kv_seq_stride_bytes, ctx_len_dev,
                                    digest_dev, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int pi_build_digests_all(pi_ctx* ctx, int batch, const void* kv, int64_t kv_seq_stride_bytes,
+                                    const int32_t* ctx_len_dev, void* digest_all_dev, void* stream) {
+    int rc = check_call(ctx, 0, batch);
+    if (rc != PI_OK) return rc;
+    if (!kv || !ctx_len_dev || !digest_all_dev || kv_seq_stride_bytes < 0) return PI_ERR_INVALID_ARG;
+    if (!pi_aligned16(kv) || !pi_aligned16(digest_all_dev) || kv_seq_stride_bytes % 16) return PI_ERR_BAD_ALIGN;
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, kv) != cudaSuccess) { (void)cudaGetLastError(); return PI_ERR_NOT_PINNED; }
+    const void* src = kv;
+    if (attr.type == cudaMemoryTypeHost) {
+        if (!attr.devicePointer) return PI_ERR_NOT_PINNED;
+        src = attr.devicePointer;
+    } else if (attr.type == cudaMemoryTypeUnregistered) {
+        return PI_ERR_NOT_PINNED;
+    }
+    return pi_launch_build_digests_all(ctx, batch, src, kv_seq_stride_bytes, ctx_len_dev, digest_all_dev,
+                                       static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int pi_table_init(pi_ctx* ctx, int batch, const int32_t* resident_dev, int32_t* block_table_dev,

@@ -28,6 +28,31 @@ __global__ void build_digests_kernel(const __nv_bfloat16* kv, long long seq_stri
     out[PI_HEAD_DIM] = hi;
 }
 
+// The same for every KV head: digest_all [batch][NB][Hkv][2][D] (the layout the averaged and
+// headwise selection strategies read).  One thread per (block, head, channel).
+__global__ void build_digests_all_kernel(const __nv_bfloat16* kv, long long seq_stride_elems, const int32_t* ctx_len,
+                                         __nv_bfloat16* digest, int Hkv, int B, int max_blocks) {
+    const int seq = blockIdx.y;
+    const int per_cta = blockDim.x / PI_HEAD_DIM;
+    const int item = blockIdx.x * per_cta + threadIdx.x / PI_HEAD_DIM;       // (block, head)
+    const int b = item / Hkv, h = item - b * Hkv;
+    const int d = threadIdx.x % PI_HEAD_DIM;
+    const int ctx = max(ctx_len[seq], 0);
+    const int n_blocks = min((ctx + B - 1) / B, max_blocks);
+    if (b >= n_blocks) return;
+    const int valid = min(B, ctx - b * B);
+    const __nv_bfloat16* k = kv + seq * seq_stride_elems + (static_cast<long long>(b) * Hkv + h) * 2ll * B * PI_HEAD_DIM + d;
+    __nv_bfloat16 lo = k[0], hi = k[0];
+    for (int t = 1; t < valid; ++t) {
+        const __nv_bfloat16 x = k[static_cast<size_t>(t) * PI_HEAD_DIM];
+        if (__bfloat162float(x) < __bfloat162float(lo)) lo = x;
+        if (__bfloat162float(x) > __bfloat162float(hi)) hi = x;
+    }
+    __nv_bfloat16* out = digest + ((static_cast<size_t>(seq) * max_blocks + b) * Hkv + h) * 2 * PI_HEAD_DIM + d;
+    out[0] = lo;
+    out[PI_HEAD_DIM] = hi;
+}
+
 __global__ void table_init_kernel(const int32_t* resident, int32_t* table, int32_t* slot_block, uint32_t* slot_stamp,
                                   int C, int max_blocks) {
     const int seq = blockIdx.x;
@@ -52,6 +77,18 @@ int pi_launch_build_digests(pi_ctx* c, int h_star, int batch, const void* kv, in
     build_digests_kernel<<<grid, threads, 0, stream>>>(static_cast<const __nv_bfloat16*>(kv), stride / 2, ctx_len,
                                                        static_cast<__nv_bfloat16*>(digest), h_star,
                                                        c->cfg.n_kv_heads, c->cfg.block_tokens, c->cfg.max_blocks);
+    PI_CUDA_TRY(cudaGetLastError());
+    return PI_OK;
+}
+
+int pi_launch_build_digests_all(pi_ctx* c, int batch, const void* kv, int64_t stride, const int32_t* ctx_len,
+                                void* digest_all, cudaStream_t stream) {
+    const int threads = 256, per_cta = threads / PI_HEAD_DIM;
+    const int items = c->cfg.max_blocks * c->cfg.n_kv_heads;
+    dim3 grid((items + per_cta - 1) / per_cta, batch);
+    build_digests_all_kernel<<<grid, threads, 0, stream>>>(static_cast<const __nv_bfloat16*>(kv), stride / 2, ctx_len,
+                                                           static_cast<__nv_bfloat16*>(digest_all), c->cfg.n_kv_heads,
+                                                           c->cfg.block_tokens, c->cfg.max_blocks);
     PI_CUDA_TRY(cudaGetLastError());
     return PI_OK;
 }

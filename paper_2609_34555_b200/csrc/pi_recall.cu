@@ -29,6 +29,7 @@ struct RecallParams {
     const int32_t* count;
     pi_status_ref st;
     long long host_stride, pool_stride, unit_bytes;
+    long long unit_stride, list_offset;            // distance between consecutive units; byte offset of list (l % lists_per_seq)
     int n_lists, lists_per_seq, cap, cache_cap;
 };
 
@@ -152,8 +153,9 @@ recall_kernel(RecallParams p) {
             continue;
         }
         const int seq = l / p.lists_per_seq;
-        const unsigned char* src = p.host + seq * p.host_stride + (static_cast<long long>(e.src_unit) + k) * p.unit_bytes + in_unit + lane * 16;
-        unsigned char* dst = p.pool + seq * p.pool_stride + (static_cast<long long>(e.dst_unit) + k) * p.unit_bytes + in_unit + lane * 16;
+        const long long loff = (l - seq * p.lists_per_seq) * p.list_offset + in_unit + lane * 16;
+        const unsigned char* src = p.host + seq * p.host_stride + (static_cast<long long>(e.src_unit) + k) * p.unit_stride + loff;
+        unsigned char* dst = p.pool + seq * p.pool_stride + (static_cast<long long>(e.dst_unit) + k) * p.unit_stride + loff;
         uint4 v[LOADS_PER_LANE];
 #pragma unroll
         for (int i = 0; i < LOADS_PER_LANE; ++i) v[i] = ld_host16(src + i * 512);
@@ -166,13 +168,16 @@ recall_kernel(RecallParams p) {
 
 int pi_launch_recall(pi_ctx* c, int n_lists, int lists_per_seq, const void* host_kv, int64_t host_stride,
                      void* pool, int64_t pool_stride, const pi_extent* list, int32_t cap,
-                     const int32_t* count, int64_t unit_bytes, cudaStream_t stream) {
+                     const int32_t* count, int64_t unit_bytes, int64_t unit_stride, int64_t list_offset,
+                     cudaStream_t stream) {
     RecallParams p;
     p.host = static_cast<const unsigned char*>(host_kv);
     p.pool = static_cast<unsigned char*>(pool);
     p.list = list; p.count = count;
     p.st = pi_status_of(c);
     p.host_stride = host_stride; p.pool_stride = pool_stride; p.unit_bytes = unit_bytes;
+    p.unit_stride = unit_stride > 0 ? unit_stride : unit_bytes;
+    p.list_offset = list_offset;
     p.n_lists = n_lists; p.lists_per_seq = lists_per_seq; p.cap = cap;
     // shared memory: two prefix arrays over the lists + the extent cache
     const long long want = static_cast<long long>(n_lists) * cap;

@@ -37,7 +37,13 @@ struct SelParams {
     unsigned int* counters;
     pi_status_ref st;
     int h_star, Hq, G, B, K, n_sink, n_local, max_blocks;
-    int batch, per;                                // sequences in the launch, chunks per CTA
+    int batch, per;                                // (virtual) sequences in the launch, chunks per CTA
+    // Which KV heads are scored.  A "virtual sequence" v is (sequence v / vh, slice v % vh); its score
+    // sums n_sum heads starting at h_base + (v % vh) * hv_step; digests hold dig_heads heads per block.
+    //   retrieval head only: vh 1, n_sum 1, h_base = that head, dig_heads 1
+    //   averaged:            vh 1, n_sum Hkv, h_base 0,         dig_heads Hkv
+    //   headwise:            vh Hkv, n_sum 1, h_base 0, hv_step 1, dig_heads Hkv
+    int vh, n_sum, h_base, hv_step, dig_heads;
 };
 
 // Shared arrays that one thread walks with a stride of several words are stored with one
@@ -251,8 +257,10 @@ __device__ __forceinline__ void select_sequence(const SelParams& p, int seq, int
 // equal runs to the CTAs; the grid is sized to what is resident at once (two CTAs per SM), so
 // small workloads get one chunk per CTA and large ones loop.  Warps run through their run
 // without CTA barriers; a barrier and a ticket follow only when the CTA leaves a sequence.
+template <bool MULTI>                              // MULTI: head sets / all-head digests (the comparison strategies)
 __global__ void __launch_bounds__(SCORE_THREADS, 2)
 score_select_kernel(SelParams p) {
+    const int vh = MULTI ? p.vh : 1, n_sum = MULTI ? p.n_sum : 1, dig_heads = MULTI ? p.dig_heads : 1;
     extern __shared__ uint32_t keys[];             // [padded(n_blocks)] in the selecting CTA
     __shared__ unsigned hist[BINS + BINS / 32 + 1];
     __shared__ unsigned warp_tot[SCORE_WARPS];
@@ -269,28 +277,35 @@ score_select_kernel(SelParams p) {
     int f = blockIdx.x * p.per;
 
     while (f < f1) {
-        const int seq = f / n_chunks;
+        const int seq = f / n_chunks;                          // virtual sequence
         const int fe = min(f1, (seq + 1) * n_chunks);          // this CTA's chunks of this sequence
-        const uint4* dg = p.digest + static_cast<size_t>(seq) * p.max_blocks * 32;   // 32 uint4 per block
+        const int rseq = seq / vh, head0 = p.h_base + (seq - rseq * vh) * p.hv_step;
         float w[8];
         int n_blocks = 0;
         for (int c = f; c < fe; ++c) {
+            const int b0 = (c - seq * n_chunks) * SCORE_CHUNK + warp * BLOCKS_PER_WARP;
+            float acc[BLOCKS_PER_WARP];
+#pragma unroll
+            for (int i = 0; i < BLOCKS_PER_WARP; ++i) acc[i] = 0.f;
+          for (int hh = 0; hh < n_sum; ++hh) {
+            const int head = head0 + hh;
             // every load is issued before anything waits: digest rows up to max_blocks are
             // allocated, so they are read unguarded and masked at the store
-            const int b0 = (c - seq * n_chunks) * SCORE_CHUNK + warp * BLOCKS_PER_WARP;
+            const uint4* dg = p.digest + (static_cast<size_t>(rseq) * p.max_blocks * dig_heads +
+                                          (dig_heads > 1 ? head : 0)) * 32;            // 32 uint4 per (block, head)
             uint4 v[BLOCKS_PER_WARP];
 #pragma unroll
             for (int i = 0; i < BLOCKS_PER_WARP; ++i) {
                 v[i] = make_uint4(0, 0, 0, 0);
-                if (b0 + i < p.max_blocks) v[i] = ld_stream16(dg + static_cast<size_t>(b0 + i) * 32 + lane);
+                if (b0 + i < p.max_blocks) v[i] = ld_stream16(dg + static_cast<size_t>(b0 + i) * dig_heads * 32 + lane);
             }
-            if (c == f) {
+            if (c == f || n_sum > 1) {
                 // lanes 0-15 hold Q- for channels 8*lane.., lanes 16-31 hold Q+ for channels 8*(lane-16)..
 #pragma unroll
                 for (int i = 0; i < 8; ++i) w[i] = 0.f;
                 const int d0 = (lane & 15) * 8;
                 const bool plus = lane >= 16;
-                const __nv_bfloat16* qh = p.q + (static_cast<size_t>(seq) * p.Hq + static_cast<size_t>(p.h_star) * p.G) * PI_HEAD_DIM + d0;
+                const __nv_bfloat16* qh = p.q + (static_cast<size_t>(rseq) * p.Hq + static_cast<size_t>(head) * p.G) * PI_HEAD_DIM + d0;
                 // the group's query rows are fetched four at a time so their latencies overlap
                 for (int g0 = 0; g0 < p.G; g0 += 4) {
                     uint4 qv[4];
@@ -310,17 +325,23 @@ score_select_kernel(SelParams p) {
                         }
                     }
                 }
-                int ctx = p.ctx_len[seq];
+            }
+            if (c == f && hh == 0) {
+                int ctx = p.ctx_len[rseq];
                 if (ctx < 0) ctx = 0;
                 n_blocks = (ctx + p.B - 1) / p.B;
                 if (n_blocks > p.max_blocks) {
-                    if (tid == 0 && c == seq * n_chunks) pi_report(p.st, PI_ERR_CAPACITY, PI_STAGE_SELECT, seq, n_blocks, p.max_blocks);
+                    if (tid == 0 && c == seq * n_chunks) pi_report(p.st, PI_ERR_CAPACITY, PI_STAGE_SELECT, rseq, n_blocks, p.max_blocks);
                     n_blocks = p.max_blocks;
                 }
             }
+#pragma unroll
+            for (int i = 0; i < BLOCKS_PER_WARP; ++i) acc[i] += dot8(v[i], w);
+          }
             float s[BLOCKS_PER_WARP];
 #pragma unroll
-            for (int i = 0; i < BLOCKS_PER_WARP; ++i) s[i] = dot8(v[i], w);
+            for (int i = 0; i < BLOCKS_PER_WARP; ++i) s[i] = acc[i];
+
             // transposed warp reduction: 8 values x 32 lanes -> lane group (lane>>2) owns block (lane>>2)
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -390,7 +411,37 @@ int pi_launch_score_select(pi_ctx* c, int h_star, int batch, const void* q, cons
     p.n_sink = c->cfg.n_sink_blocks;
     p.n_local = c->cfg.n_local_blocks;
     p.max_blocks = c->cfg.max_blocks;
+    p.vh = 1; p.n_sum = 1; p.h_base = h_star; p.hv_step = 0; p.dig_heads = 1;
     return launch_score_select(p, batch, c->n_sms, stream);
+}
+
+// The comparison strategies of the paper's selection study: averaged scores shared by all heads,
+// or one selection per KV head.  Same kernel over digests of every KV head.
+int pi_launch_score_select_strategy(pi_ctx* c, int strategy, int batch, const void* q, const void* digest_all,
+                                    const int32_t* ctx_len, int32_t* sel, int32_t* sel_count, float* scores,
+                                    unsigned int* counters, cudaStream_t stream) {
+    SelParams p;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.digest = static_cast<const uint4*>(digest_all);
+    p.ctx_len = ctx_len;
+    p.sel = sel;
+    p.sel_count = sel_count;
+    p.scores = scores;
+    p.counters = counters;
+    p.st = pi_status_of(c);
+    p.h_star = 0;
+    p.Hq = c->cfg.n_q_heads;
+    p.G = c->cfg.n_q_heads / c->cfg.n_kv_heads;
+    p.B = c->cfg.block_tokens;
+    p.K = c->cfg.budget_blocks;
+    p.n_sink = c->cfg.n_sink_blocks;
+    p.n_local = c->cfg.n_local_blocks;
+    p.max_blocks = c->cfg.max_blocks;
+    p.dig_heads = c->cfg.n_kv_heads;
+    p.h_base = 0;
+    if (strategy == PI_SELECT_AVERAGE) { p.vh = 1; p.n_sum = c->cfg.n_kv_heads; p.hv_step = 0; }
+    else { p.vh = c->cfg.n_kv_heads; p.n_sum = 1; p.hv_step = 1; }
+    return launch_score_select(p, batch * p.vh, c->n_sms, stream);
 }
 
 // Grid sizing shared by both entry points: as many CTAs as are resident at once (two per SM),
@@ -402,9 +453,11 @@ static int launch_score_select(SelParams& p, int batch, int n_sms, cudaStream_t 
     p.per = (total + 2 * n_sms - 1) / (2 * n_sms);
     const int grid = (total + p.per - 1) / p.per;
     const size_t smem = (static_cast<size_t>(p.max_blocks) + p.max_blocks / 32 + 1) * sizeof(uint32_t);
+    const bool multi = p.vh > 1 || p.n_sum > 1 || p.dig_heads > 1;
+    auto kern = multi ? score_select_kernel<true> : score_select_kernel<false>;
     if (smem > 40 * 1024)
-        PI_CUDA_TRY(cudaFuncSetAttribute(score_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    score_select_kernel<<<grid, SCORE_THREADS, smem, stream>>>(p);
+        PI_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    kern<<<grid, SCORE_THREADS, smem, stream>>>(p);
     PI_CUDA_TRY(cudaGetLastError());
     return PI_OK;
 }
@@ -486,6 +539,7 @@ extern "C" int pi_score_select_noalloc(int batch, int n_q_heads, int n_kv_heads,
     p.n_sink = n_sink_blocks;
     p.n_local = n_local_blocks;
     p.max_blocks = max_blocks;
+    p.vh = 1; p.n_sum = 1; p.h_base = solo_head; p.hv_step = 0; p.dig_heads = 1;
     // at most (8192 + 8192/32 + 1) keys: below the default dynamic shared-memory limit
     int n_sms = 0;
     PI_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));

@@ -346,3 +346,99 @@ def run_append_and_compare(cfg, steps: int, ctx_len0, layer: int = 0) -> dict:
         assert np.array_equal(host[s, :n_s], ref.kvb[s, :n_s]), "host store after the appends"
     pi.close()
     return stats
+
+
+def run_strategies_and_compare(cfg, steps: int = 2, layer: int = 0) -> dict:
+    """The averaged and the headwise selection strategies: scores and selections against the
+    oracle, then (headwise) per-head diff and per-head fragment recall, pool bytes bit-exact."""
+    from paper_2609_34555_b200 import PulseInfer
+
+    dev = torch.device("cuda:0")
+    Hkv, nb, C, K = cfg.n_kv_heads, cfg.n_blocks, cfg.pool_slots, cfg.budget_blocks
+    case = make_case(cfg, steps, layer=layer)
+    pi = PulseInfer.from_workload(cfg, max_batch=cfg.batch * Hkv)
+    ctx_d = torch.from_numpy(case.ctx_len).to(dev)
+    kvb = oracle.bits(case.kv)
+    dall = torch.zeros((cfg.batch, nb, Hkv, 2, cfg.head_dim), dtype=torch.bfloat16, device=dev)
+    pi.build_digests_all(case.kv, ctx_d, dall)
+    torch.cuda.synchronize()
+    ref_dall = np.stack([oracle.build_digest_all(kvb[s], cfg.ctx) for s in range(cfg.batch)])
+    assert np.array_equal(oracle.bits(dall.cpu()), ref_dall), "all-head digests"
+
+    # ---- averaged: one shared selection
+    sel = torch.full((cfg.batch, K), -1, dtype=torch.int32, device=dev)
+    cnt = torch.zeros((cfg.batch,), dtype=torch.int32, device=dev)
+    sc = torch.zeros((cfg.batch, nb), dtype=torch.float32, device=dev)
+    stats = dict(sel_diffs=0, misses=0)
+    for t in range(steps):
+        q_d, qb = case.q[t].to(dev), oracle.bits(case.q[t])
+        pi.score_select_strategy(pi.AVERAGE, layer, q_d, dall, ctx_d, sel, cnt, sc)
+        torch.cuda.synchronize()
+        g_sc, g_sel, g_cnt = sc.cpu().numpy(), sel.cpu().numpy(), cnt.cpu().numpy()
+        for s in range(cfg.batch):
+            want = oracle.score_heads(qb[s], ref_dall[s], nb, 0, Hkv)
+            np.testing.assert_allclose(g_sc[s], want, rtol=SCORE_RTOL, atol=SCORE_ATOL * Hkv)
+            own, own_cnt = oracle.select(g_sc[s].astype(np.float64), cfg.n_sink_blocks, cfg.n_local_blocks, K)
+            assert g_cnt[s] == own_cnt and np.array_equal(g_sel[s], own)
+            ref_sel, ref_cnt = oracle.select(want, cfg.n_sink_blocks, cfg.n_local_blocks, K)
+            gs, rs = set(g_sel[s, :ref_cnt].tolist()), set(ref_sel[:ref_cnt].tolist())
+            check_near_tie(gs, rs, want, cfg.k_mid, cfg, nb)
+            stats["sel_diffs"] += len(gs ^ rs)
+
+    # ---- headwise: every KV head selects, diffs and recalls for itself
+    R = cfg.batch * Hkv
+    hsel = torch.full((R, K), -1, dtype=torch.int32, device=dev)
+    hcnt = torch.zeros((R,), dtype=torch.int32, device=dev)
+    hsc = torch.zeros((R, nb), dtype=torch.float32, device=dev)
+    table = torch.full((R, nb), -1, dtype=torch.int32, device=dev)
+    slot_block = torch.full((R, C), -1, dtype=torch.int32, device=dev)
+    slot_stamp = torch.zeros((R, C), dtype=torch.int32, device=dev)
+    slots = torch.full((R, K), -1, dtype=torch.int32, device=dev)
+    lst = torch.zeros((R, K, 4), dtype=torch.int32, device=dev)
+    lcnt = torch.zeros((R,), dtype=torch.int32, device=dev)
+    pool = torch.zeros((cfg.batch, C, Hkv, 2, cfg.block_tokens, cfg.head_dim), dtype=torch.bfloat16, device=dev)
+    ctx_rows = ctx_d.repeat_interleave(Hkv).contiguous()
+    res_rows = np.repeat(case.resident, Hkv, axis=0)                       # every head starts with the same hot set
+    pi.table_init(torch.from_numpy(res_rows).to(dev), table, slot_block, slot_stamp)
+    # oracle state per (sequence, head)
+    o_table = np.full((R, nb), -1, np.int32)
+    o_sb = res_rows.copy()
+    o_st = np.zeros((R, C), np.uint32)
+    o_pool = np.zeros((cfg.batch, C) + kvb.shape[2:], np.uint16)
+    for r in range(R):
+        ok = res_rows[r] >= 0
+        o_table[r, res_rows[r][ok]] = np.nonzero(ok)[0]
+    frag, blockb = cfg.frag_bytes, cfg.block_bytes
+    for t in range(steps):
+        step = t + 1
+        q_d, qb = case.q[t].to(dev), oracle.bits(case.q[t])
+        pi.score_select_strategy(pi.HEADWISE, layer, q_d, dall, ctx_d, hsel, hcnt, hsc)
+        pi.diff_misses(layer, step, ctx_rows, hsel, hcnt, table, slot_block, slot_stamp, slots, lst, lcnt)
+        pi.recall_gather_scatter(layer, case.kv, pool, lst, lcnt, lists_per_seq=Hkv, unit_bytes=frag,
+                                 unit_stride=blockb, list_offset=frag)
+        torch.cuda.synchronize()
+        assert pi.status()[0] == 0, pi.status()
+        g_sc, g_sel, g_cnt = hsc.cpu().numpy(), hsel.cpu().numpy(), hcnt.cpu().numpy()
+        g_slots, g_lst, g_lcnt = slots.cpu().numpy(), lst.cpu().numpy(), lcnt.cpu().numpy()
+        for s in range(cfg.batch):
+            for h in range(Hkv):
+                r = s * Hkv + h
+                want = oracle.score_heads(qb[s], ref_dall[s], nb, h, h + 1)
+                np.testing.assert_allclose(g_sc[r], want, rtol=SCORE_RTOL, atol=SCORE_ATOL)
+                own, own_cnt = oracle.select(g_sc[r].astype(np.float64), cfg.n_sink_blocks, cfg.n_local_blocks, K)
+                assert g_cnt[r] == own_cnt and np.array_equal(g_sel[r], own)
+                ref_sel, ref_cnt = oracle.select(want, cfg.n_sink_blocks, cfg.n_local_blocks, K)
+                check_near_tie(set(g_sel[r, :ref_cnt].tolist()), set(ref_sel[:ref_cnt].tolist()), want, cfg.k_mid, cfg, nb)
+                rc, o_slots, pairs = oracle.diff(g_sel[r], int(g_cnt[r]), nb, cfg.n_sink_blocks, cfg.n_local_blocks, step,
+                                                 o_table[r], o_sb[r], o_st[r])
+                assert rc == 0 and np.array_equal(g_slots[r], o_slots)
+                assert np.array_equal(expand_extents(g_lst[r], int(g_lcnt[r])), pairs.reshape(-1, 2))
+                oracle.recall_strided(kvb[s].view(np.uint8).reshape(-1), o_pool[s].view(np.uint8).reshape(-1), pairs,
+                                      frag, blockb, h * frag)
+                stats["misses"] += len(pairs)
+        assert np.array_equal(table.cpu().numpy(), o_table)
+        assert np.array_equal(oracle.bits(pool.cpu()), o_pool), "per-head fragments in the pool"
+    # heads really choose differently (the fragmentation the shared selection avoids)
+    stats["distinct_head_selections"] = len({tuple(g_sel[h].tolist()) for h in range(Hkv)})
+    pi.close()
+    return stats

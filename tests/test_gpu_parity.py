@@ -268,3 +268,16 @@ def test_largest_supported_block_count_and_wide_budget():
     case = make_case(cfg, steps=2)
     stats = run_and_compare(case, steps=2)
     assert stats["misses"][0] > 100
+
+
+def test_averaged_and_headwise_selection_strategies():
+    from tests.parity import run_strategies_and_compare
+    cfg = tiny_config(batch=2, ctx=3000, n_q_heads=16, n_kv_heads=4, budget_blocks=32, resident_frac=0.3)
+    stats = run_strategies_and_compare(cfg, steps=2)
+    assert stats["misses"] > 0 and stats["distinct_head_selections"] > 1
+
+
+def test_strategies_with_eight_kv_heads_and_group_of_eight():
+    from tests.parity import run_strategies_and_compare
+    cfg = tiny_config(batch=2, ctx=2500, n_q_heads=64, n_kv_heads=8, budget_blocks=24, resident_frac=0.25)
+    run_strategies_and_compare(cfg, steps=2)
