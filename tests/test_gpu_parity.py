@@ -281,3 +281,42 @@ def test_strategies_with_eight_kv_heads_and_group_of_eight():
     from tests.parity import run_strategies_and_compare
     cfg = tiny_config(batch=2, ctx=2500, n_q_heads=64, n_kv_heads=8, budget_blocks=24, resident_frac=0.25)
     run_strategies_and_compare(cfg, steps=2)
+
+
+def test_group_of_sixteen_query_heads_per_kv_head():
+    """G = 16 takes the two-column-tile variant of the attention kernel."""
+    from tests.parity import make_case, run_and_compare
+    cfg = tiny_config(batch=2, ctx=2000, n_q_heads=32, n_kv_heads=2, budget_blocks=24, resident_frac=0.3)
+    run_and_compare(make_case(cfg, steps=3), steps=3)
+
+
+def test_single_kv_head_and_pure_topk_without_sink_or_local_window():
+    from tests.parity import make_case, run_and_compare
+    cfg = tiny_config(batch=2, ctx=1500, n_q_heads=4, n_kv_heads=1, budget_blocks=20, resident_frac=0.4,
+                      sink_tokens=0, local_tokens=0)
+    assert cfg.n_sink_blocks == 0 and cfg.n_local_blocks == 0 and cfg.k_mid == 20
+    # the ragged last block is then an ordinary candidate: it may or may not be selected
+    run_and_compare(make_case(cfg, steps=4, ctx_len=np.asarray([1500, 1493])), steps=4)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_shapes(seed):
+    """Randomly drawn small shapes: head counts, block sizes, budgets, pool sizes, ragged contexts."""
+    from tests.parity import make_case, run_and_compare
+    rng = np.random.default_rng(1000 + seed)
+    Hkv = int(rng.choice([1, 2, 4, 8]))
+    G = int(rng.choice([1, 2, 4, 8, 16]))
+    B = int(rng.choice([16, 32, 64]))
+    batch = int(rng.integers(1, 5))
+    nb = int(rng.integers(12, 90))
+    sink = int(rng.choice([0, 16]))
+    local = int(rng.choice([0, 128]))
+    pinned = (-(-sink // B) if sink else 0) + (max(1, local // B) if local else 0)
+    K = int(rng.integers(pinned + 1, pinned + 30))
+    cfg = tiny_config(batch=batch, ctx=nb * B - int(rng.integers(0, B)), n_q_heads=Hkv * G, n_kv_heads=Hkv,
+                      block_tokens=B, budget_blocks=K, resident_frac=float(rng.uniform(0.1, 0.9)),
+                      sink_tokens=sink, local_tokens=local, seed=seed)
+    lens = [int(rng.integers(1, cfg.ctx + 1)) for _ in range(batch)]
+    lens[0] = cfg.ctx
+    case = make_case(cfg, steps=3, ctx_len=np.asarray(lens), fill=float(rng.choice([0.0, 0.5, 1.0])))
+    run_and_compare(case, steps=3, overlapped=bool(seed % 2))

@@ -29,6 +29,8 @@ class PathConfig:
     overlap: float = 0.0      # target step-to-step selection overlap (0 = independent)
     ar1: float = 0.0          # AR(1) coefficient of the query process giving `overlap`
     miss_script: str = ""     # "pareto": miss counts per (seq, layer, step) are scripted, not left to LRU
+    sink_tokens: int = 16     # always-resident prefix (0 = none: pure top-k)
+    local_tokens: int = 128   # always-resident suffix (0 = none)
     head_dim: int = 128
     seed: int = 0
 
@@ -38,12 +40,12 @@ class PathConfig:
         return _ceil_div(self.ctx, self.block_tokens)
 
     @property
-    def n_sink_blocks(self) -> int:       # 16 sink tokens
-        return _ceil_div(16, self.block_tokens)
+    def n_sink_blocks(self) -> int:       # 16 sink tokens by default
+        return _ceil_div(self.sink_tokens, self.block_tokens) if self.sink_tokens > 0 else 0
 
     @property
-    def n_local_blocks(self) -> int:      # 128 local tokens
-        return max(1, 128 // self.block_tokens)
+    def n_local_blocks(self) -> int:      # 128 local tokens by default
+        return max(1, self.local_tokens // self.block_tokens) if self.local_tokens > 0 else 0
 
     @property
     def k_mid(self) -> int:
