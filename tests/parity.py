@@ -194,7 +194,8 @@ def run_and_compare(case: Case, steps: int, layer: int = 0, overlapped: bool = F
     return stats
 
 
-def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, settle_cold: bool = True) -> dict:
+def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, settle_cold: bool = True,
+                        append: bool = False, ctx_start: int = 0) -> dict:
     """The bench's launch configuration (DecodeSession: whole batch per call, every layer,
     three-stream pipeline) at a full-size shape; the oracle follows only `sample_seqs`, which is
     enough because sequences are independent.  Inputs are generated on the GPU and handed to the
@@ -205,40 +206,64 @@ def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, s
     dev = torch.device("cuda:0")
     pi = PulseInfer.from_workload(cfg)
     sess = DecodeSession(pi, cfg.batch, cfg.n_layers, keep_scores=True)
-    sess.ctx_len.fill_(cfg.ctx)
+    ctx_now = ctx_start or cfg.ctx                     # runs that append start short of the full context
+    sess.ctx_len.fill_(ctx_now)
+    short = cfg.replace(ctx=ctx_now)
     residents = []
     for l in range(cfg.n_layers):
         kv = gen.make_kv(cfg, l, device=dev)
-        res = gen.initial_resident(cfg, l)
+        res = np.full((cfg.batch, cfg.pool_slots), -1, np.int32)
+        r0 = gen.initial_resident(short, l)[:, :cfg.pool_slots]
+        res[:, :r0.shape[1]] = r0
         residents.append(res)
         sess.load_layer(l, kv, torch.from_numpy(res).to(dev))
         del kv
     q_all = torch.stack([gen.make_queries(cfg, l, steps, device=dev) for l in range(cfg.n_layers)], 1).contiguous()
+    new_kv = None
+    if append:
+        g = torch.Generator(device=dev).manual_seed(gen.seed_for(cfg, 98))
+        shp = (steps, cfg.n_layers, cfg.batch, cfg.n_kv_heads, cfg.head_dim)
+        new_kv = (torch.randn(shp, device=dev, generator=g).to(torch.bfloat16),
+                  torch.randn(shp, device=dev, generator=g).to(torch.bfloat16))
     torch.cuda.synchronize()
 
-    # oracle state for the sampled sequences
+    # oracle state for the sampled sequences (its own copy of the host store when tokens are appended)
     ora = {}
     for l in range(cfg.n_layers):
         kvb = oracle.bits(sess.host_region(l))
+        blk_shape = kvb.shape[2:]
+        if append:
+            kvb = {s_: kvb[s_].copy() for s_ in sample_seqs}
         h = cfg.solo_head(l)
         for s in sample_seqs:
             table = np.full(cfg.n_blocks, -1, np.int32)
             ok = residents[l][s] >= 0
             table[residents[l][s][ok]] = np.nonzero(ok)[0]
-            pool = np.zeros((cfg.pool_slots,) + kvb.shape[2:], np.uint16)
-            pool[ok] = kvb[s, residents[l][s][ok]]
-            dg = oracle.build_digest(kvb[s], cfg.ctx, h)
-            assert np.array_equal(oracle.bits(sess.bufs[l].digest[s].cpu()), dg), "digest"
+            pool = np.zeros((cfg.pool_slots,) + blk_shape, np.uint16)
+            pool[ok] = kvb[s][residents[l][s][ok]]
+            dg = oracle.build_digest(kvb[s], ctx_now, h)
+            n0 = -(-ctx_now // cfg.block_tokens)
+            assert np.array_equal(oracle.bits(sess.bufs[l].digest[s].cpu())[:n0], dg[:n0]), "digest"
             assert np.array_equal(oracle.bits(sess.bufs[l].pool[s].cpu()), pool), "initial pool"
             ora[(l, s)] = dict(kvb=kvb[s], h=h, digest=dg, table=table, slot_block=residents[l][s].copy(),
                                slot_stamp=np.zeros(cfg.pool_slots, np.uint32), pool=pool)
     stats = dict(max_abs=0.0, misses=0, sel_diffs=0)
     unit = cfg.block_bytes
     for t in range(steps):
-        sess.decode_step(q_all[t], overlapped=overlapped)
+        sess.decode_step(q_all[t], overlapped=overlapped, new_kv=(new_kv[0][t], new_kv[1][t]) if append else None)
         torch.cuda.synchronize()
         assert pi.status()[0] == 0, pi.status()
         out = sess.out.float().cpu().numpy().astype(np.float64)
+        if append:
+            for l in range(cfg.n_layers):
+                kb, vb = oracle.bits(new_kv[0][t, l].cpu()), oracle.bits(new_kv[1][t, l].cpu())
+                for s in sample_seqs:
+                    o = ora[(l, s)]
+                    rc = oracle.append(kb[s], vb[s], ctx_now, cfg.block_tokens, o["h"], cfg.n_sink_blocks, cfg.n_local_blocks,
+                                       t + 1, o["kvb"], o["pool"], o["table"], o["slot_block"], o["slot_stamp"], o["digest"])
+                    assert rc == 0
+            ctx_now += 1
+        n_now = -(-ctx_now // cfg.block_tokens)
         for l in range(cfg.n_layers):
             b = sess.bufs[l]
             g_sel, g_cnt = b.sel_blocks.cpu().numpy(), b.sel_count.cpu().numpy()
@@ -247,22 +272,22 @@ def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, s
             for s in sample_seqs:
                 o = ora[(l, s)]
                 qb = oracle.bits(q_all[t, l, s].cpu())
-                sc = oracle.score(qb, o["digest"], cfg.n_blocks, cfg.n_kv_heads, o["h"])
-                np.testing.assert_allclose(g_scores[s], sc, rtol=SCORE_RTOL, atol=SCORE_ATOL)
-                own, own_cnt = oracle.select(g_scores[s].astype(np.float64), cfg.n_sink_blocks, cfg.n_local_blocks,
+                sc = oracle.score(qb, o["digest"], n_now, cfg.n_kv_heads, o["h"])
+                np.testing.assert_allclose(g_scores[s, :n_now], sc, rtol=SCORE_RTOL, atol=SCORE_ATOL)
+                own, own_cnt = oracle.select(g_scores[s, :n_now].astype(np.float64), cfg.n_sink_blocks, cfg.n_local_blocks,
                                              cfg.budget_blocks)
                 assert g_cnt[s] == own_cnt and np.array_equal(g_sel[s], own)
                 sel_ref, cnt_ref = oracle.select(sc, cfg.n_sink_blocks, cfg.n_local_blocks, cfg.budget_blocks)
                 gs, rs = set(g_sel[s, :cnt_ref].tolist()), set(sel_ref[:cnt_ref].tolist())
-                check_near_tie(gs, rs, sc, cfg.k_mid, cfg, cfg.n_blocks)
+                check_near_tie(gs, rs, sc, cfg.k_mid, cfg, n_now)
                 stats["sel_diffs"] += len(gs ^ rs)
-                rc, slots, pairs = oracle.diff(g_sel[s], int(g_cnt[s]), cfg.n_blocks, cfg.n_sink_blocks,
+                rc, slots, pairs = oracle.diff(g_sel[s], int(g_cnt[s]), n_now, cfg.n_sink_blocks,
                                                cfg.n_local_blocks, t + 1, o["table"], o["slot_block"], o["slot_stamp"])
                 assert rc == 0 and np.array_equal(g_slots[s], slots)
                 assert np.array_equal(expand_extents(g_list[s], int(g_lcnt[s])), pairs.reshape(-1, 2))
                 oracle.recall(o["kvb"].view(np.uint8).reshape(-1, unit), o["pool"].view(np.uint8).reshape(-1, unit), pairs, unit)
                 stats["misses"] += len(pairs)
-                ref, _ = oracle.attention(qb, o["pool"], slots, g_sel[s], int(g_cnt[s]), cfg.ctx, cfg.block_tokens,
+                ref, _ = oracle.attention(qb, o["pool"], slots, g_sel[s], int(g_cnt[s]), ctx_now, cfg.block_tokens,
                                           cfg.n_kv_heads)
                 err = np.abs(out[l, s] - ref)
                 stats["max_abs"] = max(stats["max_abs"], float(err.max()))
@@ -270,6 +295,12 @@ def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, s
                 assert np.array_equal(b.block_table[s].cpu().numpy(), o["table"])
                 assert np.array_equal(b.slot_stamp[s].cpu().numpy().view(np.uint32), o["slot_stamp"])
                 assert np.array_equal(oracle.bits(b.pool[s].cpu()), o["pool"]), "pool bytes"
+    if append:
+        for l in range(cfg.n_layers):
+            host = oracle.bits(sess.host_region(l))
+            for s in sample_seqs:
+                assert np.array_equal(host[s, :n_now], ora[(l, s)]["kvb"][:n_now]), "host store after the appends"
+                assert np.array_equal(oracle.bits(sess.bufs[l].digest[s].cpu())[:n_now], ora[(l, s)]["digest"][:n_now])
     pi.close()
     return stats
 

@@ -320,3 +320,12 @@ def test_random_shapes(seed):
     lens[0] = cfg.ctx
     case = make_case(cfg, steps=3, ctx_len=np.asarray(lens), fill=float(rng.choice([0.0, 0.5, 1.0])))
     run_and_compare(case, steps=3, overlapped=bool(seed % 2))
+
+
+def test_pipelined_session_with_append_on_two_layers():
+    """DecodeSession's three-stream step with a token appended to every layer each step; the
+    context crosses a block boundary on the way."""
+    from tests.parity import run_session_sampled
+    cfg = tiny_config(batch=4, ctx=4096, n_q_heads=32, n_kv_heads=8, budget_blocks=40, resident_frac=0.3, n_layers=2)
+    stats = run_session_sampled(cfg, steps=12, sample_seqs=[0, 3], append=True, ctx_start=4096 - 20)
+    assert stats["misses"] > 0
