@@ -175,3 +175,10 @@ def recall_strided(host_seq: np.ndarray, pool_seq: np.ndarray, pairs: np.ndarray
     pairs = np.ascontiguousarray(pairs, dtype=np.int32)
     lib().pio_recall_strided(_p(host_seq), _p(pool_seq), _p(pairs), len(pairs), ctypes.c_int64(unit_bytes),
                              ctypes.c_int64(unit_stride), ctypes.c_int64(offset))
+
+
+def recall_paged(arena: np.ndarray, page_table: np.ndarray, pool_seq: np.ndarray, pairs: np.ndarray, unit_bytes: int) -> None:
+    """arena uint8 [n_pages][unit_bytes]; page_table int32 [n_blocks] (logical block -> page)."""
+    pairs = np.ascontiguousarray(pairs, dtype=np.int32)
+    page_table = np.ascontiguousarray(page_table, dtype=np.int32)
+    lib().pio_recall_paged(_p(arena), _p(page_table), _p(pool_seq), _p(pairs), len(pairs), ctypes.c_int64(unit_bytes))

@@ -401,3 +401,13 @@ void pio_recall_strided(const uint8_t* host_seq, uint8_t* pool_seq, const int32_
         memcpy(pool_seq + offset + (size_t)pairs[2 * i + 1] * unit_stride,
                host_seq + offset + (size_t)pairs[2 * i] * unit_stride, (size_t)unit_bytes);
 }
+
+/* Recall from a paged host store (Sec. 4.4.2: the recalled blocks lie scattered across host
+ * memory): logical block b of the sequence is page page_table[b] of an arena of unit_bytes-long
+ * pages.  Everything else as in pio_recall. */
+void pio_recall_paged(const uint8_t* arena, const int32_t* page_table, uint8_t* pool_seq, const int32_t* pairs,
+                      int n, int64_t unit_bytes) {
+    for (int i = 0; i < n; ++i)
+        memcpy(pool_seq + (size_t)pairs[2 * i + 1] * unit_bytes,
+               arena + (size_t)page_table[pairs[2 * i]] * unit_bytes, (size_t)unit_bytes);
+}

@@ -68,3 +68,28 @@ def test_strided_recall_moves_one_head_fragment_and_nothing_else():
     mask = np.ones(pool.shape[:2], bool)
     mask[pairs[:, 1], h] = False
     assert np.array_equal(pool[mask], snap[mask])
+
+
+def test_paged_recall_reads_the_page_the_table_names_and_nothing_else():
+    """Block b of a paged store is arena page page_table[b]: the pool must hold exactly what a
+    recall from the block-major store (the arena gathered through the table) would give."""
+    rng = np.random.default_rng(8)
+    unit, nb, n_pages, C = 128, 20, 64, 9
+    arena = rng.integers(0, 256, size=(n_pages, unit), dtype=np.uint8)
+    table = rng.permutation(n_pages)[:nb].astype(np.int32)
+    pairs = np.asarray([[2, 7], [3, 0], [19, 4]], np.int32)
+    pool = rng.integers(0, 256, size=(C, unit), dtype=np.uint8)
+    snap = pool.copy()
+    oracle.recall_paged(arena, table, pool, pairs, unit)
+    for b, s in pairs:
+        assert np.array_equal(pool[s], arena[table[b]])            # written out, no call of the oracle
+    untouched = np.setdiff1d(np.arange(C), pairs[:, 1])
+    assert np.array_equal(pool[untouched], snap[untouched])
+    # the identity table is the block-major store
+    ref = snap.copy()
+    oracle.recall(arena, ref, pairs, unit)
+    ident = snap.copy()
+    oracle.recall_paged(arena, np.arange(n_pages, dtype=np.int32), ident, pairs, unit)
+    assert np.array_equal(ident, ref)
+    # distinct pages per block: the page index, not the block index, picks the bytes
+    assert not np.array_equal(pool[7], arena[2]) or table[2] == 2
