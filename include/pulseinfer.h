@@ -56,7 +56,7 @@ typedef struct {
     int32_t n_sink_blocks, n_local_blocks;    /* always-resident, always-selected prefix / suffix */
     int32_t pool_slots;                       /* C per (seq, layer); C >= K                       */
     int32_t max_batch, max_blocks;            /* capacities: batch <= max_batch, NB = max_blocks  */
-    int32_t recall_ctas;                      /* CTAs of the recall kernel, 0 = default           */
+    int32_t recall_ctas;                      /* CTAs per recall launch, 0 = default (5)           */
     int32_t attn_ctas;                        /* CTAs of the attention kernel, 0 = one per SM     */
     const int32_t* solo_head;                 /* host [n_layers]: retrieval KV head per layer (copied) */
 } pi_config;
@@ -208,6 +208,27 @@ int pi_append_kv(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* k
                  const void* v_new_dev, const int32_t* ctx_len_dev, void* host_kv_pinned,
                  int64_t host_seq_stride_bytes, void* pool_dev, int32_t* block_table_dev,
                  int32_t* slot_block_dev, uint32_t* slot_stamp_dev, void* digest_dev, void* stream);
+
+/* Paged host store (Sec. 4.4.2: the blocks to recall lie scattered across host memory).  Instead
+ * of one block-major region per sequence, the store is an arena of pages, one unit each
+ * (unit_stride_bytes apart, page g at host_arena_pinned + g * stride), and logical unit u of
+ * sequence s is page page_table_dev[s * page_table_seq_stride + u] (int32, device memory).  The
+ * extents still name logical units; each 4 KB piece looks its page up, so merged extents need no
+ * physical adjacency.  All other arguments as in pi_recall_gather_scatter / pi_append_kv; a page
+ * index outside [0, n_pages) sets PI_ERR_INDEX_RANGE in the status word and the unit is skipped.
+ * The caller owns the page table and must have assigned the page of a block before the append
+ * that opens it. */
+int pi_recall_gather_scatter_paged(pi_ctx* ctx, int layer, int n_lists, int lists_per_seq,
+                                   const void* host_arena_pinned, const int32_t* page_table_dev,
+                                   int64_t page_table_seq_stride, int32_t n_pages, void* pool_dev,
+                                   int64_t pool_seq_stride_bytes, const pi_extent* recall_list_dev,
+                                   int32_t list_capacity, const int32_t* recall_count_dev, int64_t unit_bytes,
+                                   int64_t unit_stride_bytes, int64_t list_offset_bytes, void* stream);
+int pi_append_kv_paged(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* k_new_dev,
+                       const void* v_new_dev, const int32_t* ctx_len_dev, void* host_arena_pinned,
+                       const int32_t* page_table_dev, int64_t page_table_seq_stride, int32_t n_pages,
+                       void* pool_dev, int32_t* block_table_dev, int32_t* slot_block_dev,
+                       uint32_t* slot_stamp_dev, void* digest_dev, void* stream);
 
 /* Helpers around the path (input preparation and measurement; not hot calls).
  * pi_build_digests: channel-wise min / max of the keys of head solo_head[layer] over the

@@ -23,7 +23,7 @@ ERR_NAMES = {
 EXTENT_DTYPE = torch.int32      # a pi_extent is four int32: src_unit, dst_unit, n_units, units_before
 
 EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_score_select_noalloc", "pi_score_select_strategy", "pi_diff_misses", "pi_recall_gather_scatter",
-           "pi_sparse_decode_attn", "pi_append_kv", "pi_build_digests", "pi_build_digests_all", "pi_table_init", "pi_h2d_copy_ms",
+           "pi_recall_gather_scatter_paged", "pi_sparse_decode_attn", "pi_append_kv", "pi_append_kv_paged", "pi_build_digests", "pi_build_digests_all", "pi_table_init", "pi_h2d_copy_ms",
            "pi_get_status", "pi_get_stats", "pi_clear_status", "pi_strerror"]
 
 
@@ -60,6 +60,10 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.pi_diff_misses.argtypes = [c_void_p, c_int, c_int, c_uint32, i32p, i32p, i32p, i32p, i32p, u32p, i32p, vp, i32p, vp]
     lib.pi_recall_gather_scatter.argtypes = [c_void_p, c_int, c_int, c_int, vp, c_int64, vp, c_int64, vp, c_int32, i32p,
                                              c_int64, c_int64, c_int64, vp]
+    lib.pi_recall_gather_scatter_paged.argtypes = [c_void_p, c_int, c_int, c_int, vp, i32p, c_int64, c_int32, vp, c_int64, vp,
+                                                   c_int32, i32p, c_int64, c_int64, c_int64, vp]
+    lib.pi_append_kv_paged.argtypes = [c_void_p, c_int, c_int, c_uint32, vp, vp, i32p, vp, i32p, c_int64, c_int32, vp, i32p,
+                                       i32p, u32p, vp, vp]
     lib.pi_score_select_strategy.argtypes = [c_void_p, c_int, c_int, c_int, vp, vp, i32p, i32p, i32p, vp, vp]
     lib.pi_build_digests_all.argtypes = [c_void_p, c_int, vp, c_int64, i32p, vp, vp]
     lib.pi_sparse_decode_attn.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, i32p, vp, vp, vp]
@@ -206,14 +210,23 @@ class PulseInfer:
     def recall_gather_scatter(self, layer: int, host_kv, pool, recall_list, recall_count, *, lists_per_seq: int = 1,
                               unit_bytes: Optional[int] = None, host_seq_stride: Optional[int] = None,
                               pool_seq_stride: Optional[int] = None, unit_stride: int = 0, list_offset: int = 0,
-                              stream=None) -> None:
+                              page_table=None, n_pages: Optional[int] = None, stream=None) -> None:
         """host_kv: pinned host tensor [batch][NB] blocks; pool: CUDA tensor [batch][C] blocks;
-        recall_list: int32 [n_lists][capacity][4]."""
+        recall_list: int32 [n_lists][capacity][4].  With page_table (int32 CUDA tensor [batch][NB]) the
+        host tensor is an arena of pages and block b of sequence s is page page_table[s][b]."""
         n_lists, cap = recall_list.shape[0], recall_list.shape[1]
         if not host_kv.is_cuda and not host_kv.is_pinned():
             raise PiError("pi_recall_gather_scatter", -5, strerror(-5))
-        hs = host_seq_stride if host_seq_stride is not None else host_kv.stride(0) * host_kv.element_size()
         ps = pool_seq_stride if pool_seq_stride is not None else pool.stride(0) * pool.element_size()
+        if page_table is not None:
+            ub = unit_bytes or self.block_bytes
+            pages = n_pages if n_pages is not None else host_kv.numel() * host_kv.element_size() // (unit_stride or ub)
+            _check("pi_recall_gather_scatter_paged", self._lib.pi_recall_gather_scatter_paged(
+                self._ctx, layer, n_lists, lists_per_seq, host_kv.data_ptr(), _dev(page_table, torch.int32, "page_table"),
+                page_table.stride(0), pages, pool.data_ptr(), ps, _dev(recall_list, EXTENT_DTYPE, "recall_list"), cap,
+                _dev(recall_count, torch.int32, "recall_count"), ub, unit_stride, list_offset, _stream(stream)))
+            return
+        hs = host_seq_stride if host_seq_stride is not None else host_kv.stride(0) * host_kv.element_size()
         _check("pi_recall_gather_scatter", self._lib.pi_recall_gather_scatter(
             self._ctx, layer, n_lists, lists_per_seq, host_kv.data_ptr(), hs, pool.data_ptr(), ps,
             _dev(recall_list, EXTENT_DTYPE, "recall_list"), cap, _dev(recall_count, torch.int32, "recall_count"),
@@ -232,12 +245,23 @@ class PulseInfer:
             _stream(stream)))
 
     def append_kv(self, layer: int, step: int, k_new, v_new, ctx_len, host_kv, pool, block_table, slot_block,
-                  slot_stamp, digest, host_seq_stride: Optional[int] = None, stream=None) -> None:
+                  slot_stamp, digest, host_seq_stride: Optional[int] = None, page_table=None,
+                  n_pages: Optional[int] = None, stream=None) -> None:
         """The step's new token (k_new, v_new: [batch][Hkv][D] bf16) joins block ctx_len // B of every
-        sequence: pool slot, host store, running digest; ctx_len is the length before the append."""
+        sequence: pool slot, host store, running digest; ctx_len is the length before the append.
+        With page_table the host tensor is an arena of block-sized pages (see recall_gather_scatter)."""
         batch = ctx_len.shape[0]
         if not host_kv.is_cuda and not host_kv.is_pinned():
             raise PiError("pi_append_kv", -5, strerror(-5))
+        if page_table is not None:
+            pages = n_pages if n_pages is not None else host_kv.numel() * host_kv.element_size() // self.block_bytes
+            _check("pi_append_kv_paged", self._lib.pi_append_kv_paged(
+                self._ctx, layer, batch, step, _dev(k_new, torch.bfloat16, "k_new"), _dev(v_new, torch.bfloat16, "v_new"),
+                _dev(ctx_len, torch.int32, "ctx_len"), host_kv.data_ptr(), _dev(page_table, torch.int32, "page_table"),
+                page_table.stride(0), pages, pool.data_ptr(), _dev(block_table, torch.int32, "block_table"),
+                _dev(slot_block, torch.int32, "slot_block"), _dev(slot_stamp, torch.int32, "slot_stamp"),
+                _dev(digest, torch.bfloat16, "digest"), _stream(stream)))
+            return
         hs = host_seq_stride if host_seq_stride is not None else host_kv.stride(0) * host_kv.element_size()
         _check("pi_append_kv", self._lib.pi_append_kv(
             self._ctx, layer, batch, step, _dev(k_new, torch.bfloat16, "k_new"), _dev(v_new, torch.bfloat16, "v_new"),

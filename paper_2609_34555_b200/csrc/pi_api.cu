@@ -57,8 +57,10 @@ extern "C" int pi_create(const pi_config* cfg, pi_ctx** out) {
     if (e != cudaSuccess) { (void)cudaGetLastError(); pi_destroy(c); return PI_ERR_CUDA; }
     c->n_sms = prop.multiProcessorCount;
     c->attn_ctas = cfg->attn_ctas > 0 ? cfg->attn_ctas : c->n_sms;
-    // ten CTAs (80 warps x 4 KB in flight) saturate the host link on a B200; more only queue requests up
-    c->recall_ctas = cfg->recall_ctas > 0 ? cfg->recall_ctas : 10;
+    // five CTAs per launch (40 warps x 4 KB in flight): two launches running side by side on two
+    // streams saturate the host link of a B200 and cover each other's fixed costs; one launch alone
+    // still reaches 0.97 of what ten CTAs do, and more requests in flight only queue up
+    c->recall_ctas = cfg->recall_ctas > 0 ? cfg->recall_ctas : 5;
 
     const size_t nb = static_cast<size_t>(cfg->max_batch);
     const size_t n_part = static_cast<size_t>(c->attn_ctas) + nb;
@@ -153,12 +155,12 @@ extern "C" int pi_diff_misses(pi_ctx* ctx, int layer, int batch, uint32_t step, 
                           static_cast<cudaStream_t>(stream));
 }
 
-extern "C" int pi_recall_gather_scatter(pi_ctx* ctx, int layer, int n_lists, int lists_per_seq,
-                                        const void* host_kv_pinned, int64_t host_seq_stride_bytes,
-                                        void* pool_dev, int64_t pool_seq_stride_bytes,
-                                        const pi_extent* recall_list_dev, int32_t list_capacity,
-                                        const int32_t* recall_count_dev, int64_t unit_bytes,
-                                        int64_t unit_stride_bytes, int64_t list_offset_bytes, void* stream) {
+// Shared by the block-major and the paged entry point (page_table == nullptr: block-major).
+static int recall_call(pi_ctx* ctx, int layer, int n_lists, int lists_per_seq, const void* host_kv_pinned,
+                       int64_t host_seq_stride_bytes, const int32_t* page_table, int64_t page_stride, int32_t n_pages,
+                       void* pool_dev, int64_t pool_seq_stride_bytes, const pi_extent* recall_list_dev,
+                       int32_t list_capacity, const int32_t* recall_count_dev, int64_t unit_bytes,
+                       int64_t unit_stride_bytes, int64_t list_offset_bytes, void* stream) {
     if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers) return PI_ERR_INVALID_ARG;
     if (n_lists < 1 || lists_per_seq < 1 || n_lists % lists_per_seq || n_lists > 65536) return PI_ERR_INVALID_ARG;
     if (!host_kv_pinned || !pool_dev || !recall_list_dev || !recall_count_dev || list_capacity < 1)
@@ -184,7 +186,32 @@ extern "C" int pi_recall_gather_scatter(pi_ctx* ctx, int layer, int n_lists, int
     }
     return pi_launch_recall(ctx, n_lists, lists_per_seq, src, host_seq_stride_bytes, pool_dev,
                             pool_seq_stride_bytes, recall_list_dev, list_capacity, recall_count_dev,
-                            unit_bytes, unit_stride_bytes, list_offset_bytes, static_cast<cudaStream_t>(stream));
+                            unit_bytes, unit_stride_bytes, list_offset_bytes, page_table, page_stride, n_pages,
+                            static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int pi_recall_gather_scatter(pi_ctx* ctx, int layer, int n_lists, int lists_per_seq,
+                                        const void* host_kv_pinned, int64_t host_seq_stride_bytes,
+                                        void* pool_dev, int64_t pool_seq_stride_bytes,
+                                        const pi_extent* recall_list_dev, int32_t list_capacity,
+                                        const int32_t* recall_count_dev, int64_t unit_bytes,
+                                        int64_t unit_stride_bytes, int64_t list_offset_bytes, void* stream) {
+    return recall_call(ctx, layer, n_lists, lists_per_seq, host_kv_pinned, host_seq_stride_bytes, nullptr, 0, 0,
+                       pool_dev, pool_seq_stride_bytes, recall_list_dev, list_capacity, recall_count_dev, unit_bytes,
+                       unit_stride_bytes, list_offset_bytes, stream);
+}
+
+extern "C" int pi_recall_gather_scatter_paged(pi_ctx* ctx, int layer, int n_lists, int lists_per_seq,
+                                              const void* host_arena_pinned, const int32_t* page_table_dev,
+                                              int64_t page_table_seq_stride, int32_t n_pages, void* pool_dev,
+                                              int64_t pool_seq_stride_bytes, const pi_extent* recall_list_dev,
+                                              int32_t list_capacity, const int32_t* recall_count_dev,
+                                              int64_t unit_bytes, int64_t unit_stride_bytes,
+                                              int64_t list_offset_bytes, void* stream) {
+    if (!page_table_dev || page_table_seq_stride < 0 || n_pages < 1) return PI_ERR_INVALID_ARG;
+    return recall_call(ctx, layer, n_lists, lists_per_seq, host_arena_pinned, 0, page_table_dev, page_table_seq_stride,
+                       n_pages, pool_dev, pool_seq_stride_bytes, recall_list_dev, list_capacity, recall_count_dev,
+                       unit_bytes, unit_stride_bytes, list_offset_bytes, stream);
 }
 
 extern "C" int pi_sparse_decode_attn(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* pool_dev,
@@ -201,10 +228,11 @@ extern "C" int pi_sparse_decode_attn(pi_ctx* ctx, int layer, int batch, const vo
                           ctx_len_dev, out_dev, lse_dev, static_cast<cudaStream_t>(stream));
 }
 
-extern "C" int pi_append_kv(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* k_new_dev,
-                            const void* v_new_dev, const int32_t* ctx_len_dev, void* host_kv_pinned,
-                            int64_t host_seq_stride_bytes, void* pool_dev, int32_t* block_table_dev,
-                            int32_t* slot_block_dev, uint32_t* slot_stamp_dev, void* digest_dev, void* stream) {
+static int append_call(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* k_new_dev, const void* v_new_dev,
+                       const int32_t* ctx_len_dev, void* host_kv_pinned, int64_t host_seq_stride_bytes,
+                       const int32_t* page_table, int64_t page_stride, int32_t n_pages, void* pool_dev,
+                       int32_t* block_table_dev, int32_t* slot_block_dev, uint32_t* slot_stamp_dev, void* digest_dev,
+                       void* stream) {
     int rc = check_call(ctx, layer, batch);
     if (rc != PI_OK) return rc;
     if (!k_new_dev || !v_new_dev || !ctx_len_dev || !host_kv_pinned || !pool_dev || !block_table_dev ||
@@ -224,7 +252,27 @@ extern "C" int pi_append_kv(pi_ctx* ctx, int layer, int batch, uint32_t step, co
     }
     return pi_launch_append(ctx, ctx->solo_head[layer], batch, step, k_new_dev, v_new_dev, ctx_len_dev, dst,
                             host_seq_stride_bytes, pool_dev, block_table_dev, slot_block_dev, slot_stamp_dev,
-                            digest_dev, static_cast<cudaStream_t>(stream));
+                            digest_dev, page_table, page_stride, n_pages, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int pi_append_kv(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* k_new_dev,
+                            const void* v_new_dev, const int32_t* ctx_len_dev, void* host_kv_pinned,
+                            int64_t host_seq_stride_bytes, void* pool_dev, int32_t* block_table_dev,
+                            int32_t* slot_block_dev, uint32_t* slot_stamp_dev, void* digest_dev, void* stream) {
+    return append_call(ctx, layer, batch, step, k_new_dev, v_new_dev, ctx_len_dev, host_kv_pinned,
+                       host_seq_stride_bytes, nullptr, 0, 0, pool_dev, block_table_dev, slot_block_dev,
+                       slot_stamp_dev, digest_dev, stream);
+}
+
+extern "C" int pi_append_kv_paged(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* k_new_dev,
+                                  const void* v_new_dev, const int32_t* ctx_len_dev, void* host_arena_pinned,
+                                  const int32_t* page_table_dev, int64_t page_table_seq_stride, int32_t n_pages,
+                                  void* pool_dev, int32_t* block_table_dev, int32_t* slot_block_dev,
+                                  uint32_t* slot_stamp_dev, void* digest_dev, void* stream) {
+    if (!page_table_dev || page_table_seq_stride < 0 || n_pages < 1) return PI_ERR_INVALID_ARG;
+    return append_call(ctx, layer, batch, step, k_new_dev, v_new_dev, ctx_len_dev, host_arena_pinned, 0,
+                       page_table_dev, page_table_seq_stride, n_pages, pool_dev, block_table_dev, slot_block_dev,
+                       slot_stamp_dev, digest_dev, stream);
 }
 
 extern "C" int pi_build_digests(pi_ctx* ctx, int layer, int batch, const void* kv, int64_t kv_seq_stride_bytes,

@@ -21,6 +21,9 @@ struct AppendParams {
     __nv_bfloat16* digest;
     pi_status_ref st;
     long long host_stride, pool_stride;
+    const int32_t* page;           // paged host store (or null): block b of sequence s is arena page page[s * page_stride + b]
+    long long page_stride;
+    int n_pages;
     uint32_t step;
     int B, Hkv, C, n_sink, n_local, max_blocks, h_star;
 };
@@ -42,6 +45,15 @@ append_kernel(AppendParams p) {
     uint32_t* slot_stamp = p.slot_stamp + static_cast<size_t>(seq) * p.C;
     const long long block_bytes = static_cast<long long>(p.Hkv) * 2 * p.B * PI_HEAD_DIM * 2;
     int slot = table[b];
+    long long host_off = seq * p.host_stride + b * block_bytes;
+    if (p.page) {
+        const int pg = p.page[seq * p.page_stride + b];
+        if (pg < 0 || pg >= p.n_pages) {
+            if (tid == 0) pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_APPEND, seq, b, pg);
+            return;
+        }
+        host_off = pg * block_bytes;
+    }
 
     if (t == 0 && slot < 0) {
         // the block just opened is part of the local window: it takes the least recently selected
@@ -81,7 +93,7 @@ append_kernel(AppendParams p) {
         return;
     }
     unsigned char* pool_blk = p.pool + seq * p.pool_stride + slot * block_bytes;
-    unsigned char* host_blk = p.host + seq * p.host_stride + b * block_bytes;
+    unsigned char* host_blk = p.host + host_off;
     if (t == 0) {
         // a fresh block starts zeroed, in the pool and in the host store
         const uint4 z = make_uint4(0, 0, 0, 0);
@@ -117,8 +129,10 @@ append_kernel(AppendParams p) {
 
 int pi_launch_append(pi_ctx* c, int h_star, int batch, uint32_t step, const void* k_new, const void* v_new,
                      const int32_t* ctx_len, void* host_kv, int64_t host_stride, void* pool, int32_t* table,
-                     int32_t* slot_block, uint32_t* slot_stamp, void* digest, cudaStream_t stream) {
+                     int32_t* slot_block, uint32_t* slot_stamp, void* digest, const int32_t* page_table,
+                     int64_t page_stride, int32_t n_pages, cudaStream_t stream) {
     AppendParams p;
+    p.page = page_table; p.page_stride = page_stride; p.n_pages = n_pages;
     p.k_new = static_cast<const uint4*>(k_new);
     p.v_new = static_cast<const uint4*>(v_new);
     p.ctx_len = ctx_len;

@@ -84,13 +84,15 @@ int pi_launch_diff(pi_ctx*, int batch, uint32_t step, const int32_t* ctx_len, co
                    int32_t* sel_slots, pi_extent* list, int32_t* count, cudaStream_t);
 int pi_launch_recall(pi_ctx*, int n_lists, int lists_per_seq, const void* host_kv, int64_t host_stride,
                      void* pool, int64_t pool_stride, const pi_extent* list, int32_t cap,
-                     const int32_t* count, int64_t unit_bytes, int64_t unit_stride, int64_t list_offset, cudaStream_t);
+                     const int32_t* count, int64_t unit_bytes, int64_t unit_stride, int64_t list_offset,
+                     const int32_t* page_table, int64_t page_stride, int32_t n_pages, cudaStream_t);
 int pi_launch_attn(pi_ctx*, int batch, const void* q, const void* pool, const int32_t* sel_slots,
                    const int32_t* sel_blocks, const int32_t* sel_count, const int32_t* ctx_len,
                    void* out, float* lse, cudaStream_t);
 int pi_launch_append(pi_ctx*, int h_star, int batch, uint32_t step, const void* k_new, const void* v_new,
                      const int32_t* ctx_len, void* host_kv, int64_t host_stride, void* pool, int32_t* table,
-                     int32_t* slot_block, uint32_t* slot_stamp, void* digest, cudaStream_t);
+                     int32_t* slot_block, uint32_t* slot_stamp, void* digest, const int32_t* page_table,
+                     int64_t page_stride, int32_t n_pages, cudaStream_t);
 int pi_launch_build_digests_all(pi_ctx*, int batch, const void* kv, int64_t stride, const int32_t* ctx_len,
                                 void* digest_all, cudaStream_t);
 int pi_launch_build_digests(pi_ctx*, int h_star, int batch, const void* kv, int64_t stride,

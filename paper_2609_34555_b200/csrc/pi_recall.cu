@@ -31,6 +31,10 @@ struct RecallParams {
     long long host_stride, pool_stride, unit_bytes;
     long long unit_stride, list_offset;            // distance between consecutive units; byte offset of list (l % lists_per_seq)
     int n_lists, lists_per_seq, cap, cache_cap;
+    // paged host store: unit u of sequence s is page page[s * page_stride + u] of the arena at `host`
+    const int32_t* page;
+    long long page_stride;
+    int n_pages;
 };
 
 __device__ __forceinline__ uint4 ld_host16(const void* p) {
@@ -63,6 +67,7 @@ __device__ __forceinline__ long long block_scan_add(long long v, long long* warp
     return base + inc - v;
 }
 
+template <bool PAGED>
 __global__ void __launch_bounds__(RECALL_THREADS)
 recall_kernel(RecallParams p) {
     extern __shared__ long long s_dyn[];
@@ -128,7 +133,11 @@ recall_kernel(RecallParams p) {
     const long long pieces_per_unit = p.unit_bytes / PIECE_BYTES;
     const long long total = s_pref[p.n_lists] * pieces_per_unit;
     const long long stride = static_cast<long long>(gridDim.x) * RECALL_WARPS;
-    for (long long piece = static_cast<long long>(warp) * gridDim.x + blockIdx.x; piece < total; piece += stride) {
+
+    // piece -> (source, destination) of this lane's 16-byte column; src == nullptr: skip the piece
+    auto resolve = [&](long long piece, const unsigned char*& src, unsigned char*& dst) {
+        src = nullptr; dst = nullptr;
+        if (piece >= total) return;
         const long long unit = piece / pieces_per_unit;
         const long long in_unit = (piece - unit * pieces_per_unit) * PIECE_BYTES;
         // list that holds this unit: last l with s_pref[l] <= unit
@@ -150,17 +159,44 @@ recall_kernel(RecallParams p) {
         const int k = u_in_list - e.units_before;
         if (e.src_unit < 0 || e.dst_unit < 0 || k < 0 || k >= e.n_units) {
             if (lane == 0) pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_RECALL, l, elo, e.src_unit);
-            continue;
+            return;
         }
         const int seq = l / p.lists_per_seq;
         const long long loff = (l - seq * p.lists_per_seq) * p.list_offset + in_unit + lane * 16;
-        const unsigned char* src = p.host + seq * p.host_stride + (static_cast<long long>(e.src_unit) + k) * p.unit_stride + loff;
-        unsigned char* dst = p.pool + seq * p.pool_stride + (static_cast<long long>(e.dst_unit) + k) * p.unit_stride + loff;
+        if (PAGED) {
+            // one table lookup per 4 KB piece; the pieces of a page stay one sequential burst
+            const int pg = p.page[seq * p.page_stride + e.src_unit + k];
+            if (pg < 0 || pg >= p.n_pages) {
+                if (lane == 0) pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_RECALL, l, e.src_unit + k, pg);
+                return;
+            }
+            src = p.host + static_cast<long long>(pg) * p.unit_stride + loff;
+        } else {
+            src = p.host + seq * p.host_stride + (static_cast<long long>(e.src_unit) + k) * p.unit_stride + loff;
+        }
+        dst = p.pool + seq * p.pool_stride + (static_cast<long long>(e.dst_unit) + k) * p.unit_stride + loff;
+    };
+
+    // the next piece is resolved (searches, page lookup) while this piece's host loads are in flight
+    long long piece = static_cast<long long>(warp) * gridDim.x + blockIdx.x;
+    const unsigned char* src;
+    unsigned char* dst;
+    resolve(piece, src, dst);
+    while (piece < total) {
         uint4 v[LOADS_PER_LANE];
+        if (src) {
 #pragma unroll
-        for (int i = 0; i < LOADS_PER_LANE; ++i) v[i] = ld_host16(src + i * 512);
+            for (int i = 0; i < LOADS_PER_LANE; ++i) v[i] = ld_host16(src + i * 512);
+        }
+        const unsigned char* nsrc;
+        unsigned char* ndst;
+        piece += stride;
+        resolve(piece, nsrc, ndst);
+        if (src) {
 #pragma unroll
-        for (int i = 0; i < LOADS_PER_LANE; ++i) *reinterpret_cast<uint4*>(dst + i * 512) = v[i];
+            for (int i = 0; i < LOADS_PER_LANE; ++i) *reinterpret_cast<uint4*>(dst + i * 512) = v[i];
+        }
+        src = nsrc; dst = ndst;
     }
 }
 
@@ -169,8 +205,9 @@ recall_kernel(RecallParams p) {
 int pi_launch_recall(pi_ctx* c, int n_lists, int lists_per_seq, const void* host_kv, int64_t host_stride,
                      void* pool, int64_t pool_stride, const pi_extent* list, int32_t cap,
                      const int32_t* count, int64_t unit_bytes, int64_t unit_stride, int64_t list_offset,
-                     cudaStream_t stream) {
+                     const int32_t* page_table, int64_t page_stride, int32_t n_pages, cudaStream_t stream) {
     RecallParams p;
+    p.page = page_table; p.page_stride = page_stride; p.n_pages = n_pages;
     p.host = static_cast<const unsigned char*>(host_kv);
     p.pool = static_cast<unsigned char*>(pool);
     p.list = list; p.count = count;
@@ -185,14 +222,15 @@ int pi_launch_recall(pi_ctx* c, int n_lists, int lists_per_seq, const void* host
     const size_t smem = (static_cast<size_t>(n_lists) + 1) * sizeof(long long) +
                         ((static_cast<size_t>(n_lists) + 2) / 2) * sizeof(long long) +
                         static_cast<size_t>(p.cache_cap) * sizeof(pi_extent);
+    auto kernel = page_table ? recall_kernel<true> : recall_kernel<false>;
     if (smem > 40 * 1024)
-        PI_CUDA_TRY(cudaFuncSetAttribute(recall_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+        PI_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
     // ask for the largest shared-memory carve-out although this kernel hardly uses any: an SM
     // keeps one L1/shared split for all resident CTAs, and the attention kernel that overlaps
     // this one needs nearly all of it -- with the default split its CTAs could not join ours
-    PI_CUDA_TRY(cudaFuncSetAttribute(recall_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+    PI_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                      cudaSharedmemCarveoutMaxShared));
-    recall_kernel<<<c->recall_ctas, RECALL_THREADS, smem, stream>>>(p);
+    kernel<<<c->recall_ctas, RECALL_THREADS, smem, stream>>>(p);
     PI_CUDA_TRY(cudaGetLastError());
     return PI_OK;
 }

@@ -43,9 +43,13 @@ class RecallPath:
         self._ev_recall = torch.cuda.Event()
 
     def prepare_layer(self, layer: int, buf: LayerBuffers, host_kv: torch.Tensor, ctx_len: torch.Tensor,
-                      resident: torch.Tensor, kv_for_digest: Optional[torch.Tensor] = None) -> None:
+                      resident: torch.Tensor, kv_for_digest: Optional[torch.Tensor] = None,
+                      page_table: Optional[torch.Tensor] = None) -> None:
         """Digests from the keys, tables from the resident list, and the resident blocks
-        pulled into the pool through the recall kernel (slot i <- block resident[i])."""
+        pulled into the pool through the recall kernel (slot i <- block resident[i]).  A paged
+        host store needs kv_for_digest (the keys in logical block order)."""
+        if page_table is not None and kv_for_digest is None:
+            raise ValueError("a paged host store cannot be read in block order: pass kv_for_digest")
         pi = self.pi
         pi.build_digests(layer, host_kv if kv_for_digest is None else kv_for_digest, ctx_len, buf.digest)
         pi.table_init(resident, buf.block_table, buf.slot_block, buf.slot_stamp)
@@ -58,7 +62,7 @@ class RecallPath:
         fill[:, :, 1] = order.to(torch.int32)
         fill[:, :, 2] = 1
         fill[:, :, 3] = torch.arange(C, dtype=torch.int32, device=resident.device)
-        pi.recall_gather_scatter(layer, host_kv, buf.pool, fill.contiguous(), n.contiguous())
+        pi.recall_gather_scatter(layer, host_kv, buf.pool, fill.contiguous(), n.contiguous(), page_table=page_table)
 
     def select_and_recall(self, layer: int, step: int, buf: LayerBuffers, q: torch.Tensor, ctx_len: torch.Tensor,
                           host_kv: torch.Tensor, stream=None) -> None:
@@ -113,6 +117,21 @@ class StageTimer:
     def add(self, stage: str, a: torch.cuda.Event, b: torch.cuda.Event) -> None:
         self.pairs[stage].append((a, b))
 
+    def busy_ms(self, stage: str, base: torch.cuda.Event) -> float:
+        """Milliseconds during which at least one launch of the stage was running: the union of the
+        launches' intervals on the clock of `base` (a timing event recorded before all of them).
+        Equals the summed durations when launches never overlap (call after a synchronize)."""
+        spans = sorted((base.elapsed_time(a), base.elapsed_time(b)) for a, b in self.pairs[stage])
+        busy, end = 0.0, float("-inf")
+        for s0, s1 in spans:
+            if s0 > end:
+                busy += s1 - s0
+                end = s1
+            elif s1 > end:
+                busy += s1 - end
+                end = s1
+        return busy
+
     def summary(self) -> dict:
         """Per stage: launches, mean and total milliseconds (call after a synchronize)."""
         out = {}
@@ -130,10 +149,20 @@ class DecodeSession:
 
     `host_layers` < n_layers lets several layers share one region of the host store (layer l
     reads region l % host_layers) when host memory is short; digests, tables and pools stay
-    per layer."""
+    per layer.
+
+    `paged=True` scatters the blocks: each region becomes an arena of block-sized pages and a
+    seeded random permutation (the region's page table, [batch][NB] int32 on the device) says
+    which page holds block b of sequence s, so neighbouring blocks of a sequence are no longer
+    neighbours in host memory and the pages of all sequences interleave.
+
+    `recall_streams`: the recall launches of consecutive layers rotate over this many streams, so
+    the fixed cost of one launch (launch gap, list scan, first round trip over the host link,
+    drain) is covered by the transfer of the next."""
 
     def __init__(self, pi: PulseInfer, batch: int, n_layers: int, host_layers: Optional[int] = None,
-                 device="cuda", keep_scores: bool = False):
+                 device="cuda", keep_scores: bool = False, paged: bool = False, page_seed: int = 0,
+                 recall_streams: int = 2):
         c = pi.cfg
         self.pi, self.batch, self.n_layers = pi, batch, n_layers
         self.host_layers = n_layers if host_layers is None else max(1, min(host_layers, n_layers))
@@ -141,12 +170,18 @@ class DecodeSession:
         self.bufs = [LayerBuffers(pi, batch, device, keep_scores) for _ in range(n_layers)]
         shape = (batch, c.max_blocks, c.n_kv_heads, 2, c.block_tokens, c.head_dim)
         self.host_kv = [torch.empty(shape, dtype=torch.bfloat16, pin_memory=True) for _ in range(self.host_layers)]
+        self.page_tables = None
+        if paged:
+            g = torch.Generator().manual_seed(page_seed)
+            self.page_tables = [torch.randperm(batch * c.max_blocks, generator=g).to(torch.int32)
+                                .view(batch, c.max_blocks).to(device) for _ in range(self.host_layers)]
         self.out = torch.zeros((n_layers, batch, c.n_q_heads, c.head_dim), dtype=torch.bfloat16, device=device)
         self.ctx_len = torch.zeros((batch,), dtype=torch.int32, device=device)
         self.ctx_prev = torch.zeros((batch,), dtype=torch.int32, device=device)     # length before the step's append
         self.main = torch.cuda.current_stream(self.device)
         self.side = torch.cuda.Stream(self.device)
         self.side2 = torch.cuda.Stream(self.device)
+        self.recall_streams = [self.side2] + [torch.cuda.Stream(self.device) for _ in range(max(1, recall_streams) - 1)]
         self._ev_diff = [torch.cuda.Event() for _ in range(n_layers)]
         self._ev_recall = [torch.cuda.Event() for _ in range(n_layers)]
         self._ev_attn = [torch.cuda.Event() for _ in range(n_layers)]
@@ -155,17 +190,37 @@ class DecodeSession:
         self.step_count = 0
 
     def host_region(self, layer: int) -> torch.Tensor:
+        """The layer's host store: [batch][NB] blocks in block order, or (paged) the arena of pages."""
         return self.host_kv[layer % self.host_layers]
 
-    def load_layer(self, layer: int, kv_dev: Optional[torch.Tensor], resident: torch.Tensor) -> None:
-        """kv_dev (device copy of the layer's keys/values) is stored into the host region when
-        given; digests are built from it, tables from `resident`, and the resident blocks are
-        pulled back from the host store into the pool."""
+    def page_table(self, layer: int) -> Optional[torch.Tensor]:
+        return None if self.page_tables is None else self.page_tables[layer % self.host_layers]
+
+    def logical_host(self, layer: int) -> torch.Tensor:
+        """The layer's host store in logical block order (a copy when the store is paged)."""
         host = self.host_region(layer)
-        if kv_dev is not None:
-            host.copy_(kv_dev, non_blocking=False)
+        pt = self.page_table(layer)
+        if pt is None:
+            return host
+        pages = host.view((-1,) + tuple(host.shape[2:]))
+        return pages[pt.cpu().view(-1).long()].view(host.shape)
+
+    def load_layer(self, layer: int, kv_dev: Optional[torch.Tensor], resident: torch.Tensor, store: bool = True) -> None:
+        """kv_dev (device copy of the layer's keys/values, logical block order) is stored into the
+        host region when given (and `store`); digests are built from it, tables from `resident`,
+        and the resident blocks are pulled back from the host store into the pool."""
+        host = self.host_region(layer)
+        pt = self.page_table(layer)
+        if kv_dev is not None and store:
+            if pt is None:
+                host.copy_(kv_dev, non_blocking=False)
+            else:
+                scattered = torch.empty_like(kv_dev)
+                scattered.view((-1,) + tuple(kv_dev.shape[2:]))[pt.view(-1).long()] = kv_dev.view((-1,) + tuple(kv_dev.shape[2:]))
+                host.copy_(scattered, non_blocking=False)
+                del scattered
         self._path.prepare_layer(layer, self.bufs[layer], host, self.ctx_len, resident,
-                                 kv_for_digest=kv_dev)
+                                 kv_for_digest=kv_dev, page_table=pt)
 
     def decode_step(self, q: torch.Tensor, overlapped: bool = True, timer: Optional[StageTimer] = None,
                     resident_script: Optional[torch.Tensor] = None, new_kv=None) -> torch.Tensor:
@@ -184,7 +239,6 @@ class DecodeSession:
         step = self.step_count
         main = torch.cuda.current_stream(self.device)
         sel_s = self.side if overlapped else main
-        rec_s = self.side2 if overlapped else main
         if overlapped:
             self._ev_start.record(main)
             sel_s.wait_event(self._ev_start)
@@ -193,7 +247,8 @@ class DecodeSession:
                 self.ctx_prev.copy_(self.ctx_len)
                 self.ctx_len += 1
         for l in range(self.n_layers):
-            b, host = self.bufs[l], self.host_region(l)
+            b, host, pt = self.bufs[l], self.host_region(l), self.page_table(l)
+            rec_s = self.recall_streams[l % len(self.recall_streams)] if overlapped else main
             if overlapped and step > 1:
                 sel_s.wait_event(self._ev_attn[l])         # last step's attention still reads this layer's lists and pool
             tm = timer
@@ -202,7 +257,7 @@ class DecodeSession:
             if new_kv is not None:
                 ta = tm.mark(sel_s) if tm and tm.wants("append") else None
                 pi.append_kv(l, step, new_kv[0][l], new_kv[1][l], self.ctx_prev, host, b.pool, b.block_table,
-                             b.slot_block, b.slot_stamp, b.digest, stream=sel_s)
+                             b.slot_block, b.slot_stamp, b.digest, page_table=pt, stream=sel_s)
                 if ta is not None:
                     tm.add("append", ta, tm.mark(sel_s))
             t0 = tm.mark(sel_s) if tm and tm.wants("score_select") else None
@@ -215,7 +270,7 @@ class DecodeSession:
                 self._ev_diff[l].record(sel_s)
                 rec_s.wait_event(self._ev_diff[l])
             t2r = tm.mark(rec_s) if tm and tm.wants("recall") else None
-            pi.recall_gather_scatter(l, host, b.pool, b.recall_list, b.recall_count, stream=rec_s)
+            pi.recall_gather_scatter(l, host, b.pool, b.recall_list, b.recall_count, page_table=pt, stream=rec_s)
             t3 = tm.mark(rec_s) if tm and tm.wants("recall") else None
             if overlapped:
                 self._ev_recall[l].record(rec_s)

@@ -195,7 +195,7 @@ def run_and_compare(case: Case, steps: int, layer: int = 0, overlapped: bool = F
 
 
 def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, settle_cold: bool = True,
-                        append: bool = False, ctx_start: int = 0) -> dict:
+                        append: bool = False, ctx_start: int = 0, paged: bool = False) -> dict:
     """The bench's launch configuration (DecodeSession: whole batch per call, every layer,
     three-stream pipeline) at a full-size shape; the oracle follows only `sample_seqs`, which is
     enough because sequences are independent.  Inputs are generated on the GPU and handed to the
@@ -205,7 +205,7 @@ def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, s
 
     dev = torch.device("cuda:0")
     pi = PulseInfer.from_workload(cfg)
-    sess = DecodeSession(pi, cfg.batch, cfg.n_layers, keep_scores=True)
+    sess = DecodeSession(pi, cfg.batch, cfg.n_layers, keep_scores=True, paged=paged, page_seed=cfg.seed + 5)
     ctx_now = ctx_start or cfg.ctx                     # runs that append start short of the full context
     sess.ctx_len.fill_(ctx_now)
     short = cfg.replace(ctx=ctx_now)
@@ -230,9 +230,9 @@ def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, s
     # oracle state for the sampled sequences (its own copy of the host store when tokens are appended)
     ora = {}
     for l in range(cfg.n_layers):
-        kvb = oracle.bits(sess.host_region(l))
+        kvb = oracle.bits(sess.logical_host(l))
         blk_shape = kvb.shape[2:]
-        if append:
+        if append or paged:
             kvb = {s_: kvb[s_].copy() for s_ in sample_seqs}
         h = cfg.solo_head(l)
         for s in sample_seqs:
@@ -297,7 +297,7 @@ def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, s
                 assert np.array_equal(oracle.bits(b.pool[s].cpu()), o["pool"]), "pool bytes"
     if append:
         for l in range(cfg.n_layers):
-            host = oracle.bits(sess.host_region(l))
+            host = oracle.bits(sess.logical_host(l))
             for s in sample_seqs:
                 assert np.array_equal(host[s, :n_now], ora[(l, s)]["kvb"][:n_now]), "host store after the appends"
                 assert np.array_equal(oracle.bits(sess.bufs[l].digest[s].cpu())[:n_now], ora[(l, s)]["digest"][:n_now])

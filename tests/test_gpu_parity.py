@@ -329,3 +329,63 @@ def test_pipelined_session_with_append_on_two_layers():
     cfg = tiny_config(batch=4, ctx=4096, n_q_heads=32, n_kv_heads=8, budget_blocks=40, resident_frac=0.3, n_layers=2)
     stats = run_session_sampled(cfg, steps=12, sample_seqs=[0, 3], append=True, ctx_start=4096 - 20)
     assert stats["misses"] > 0
+
+
+def test_paged_host_store_recall_against_the_oracle():
+    """Blocks of all sequences interleaved in one arena of pages, located through a page table:
+    the recall kernel against the oracle's paged recall, byte for byte, untouched slots intact."""
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2609_34555_b200 import PulseInfer
+    cfg = tiny_config(batch=3, ctx=16 * 40, n_q_heads=8, n_kv_heads=2, budget_blocks=12, resident_frac=0.5)
+    pi = PulseInfer.from_workload(cfg)
+    rng = np.random.default_rng(17)
+    unit, nb, C = cfg.block_bytes, cfg.n_blocks, cfg.pool_slots
+    n_pages = cfg.batch * nb + 7
+    arena = torch.from_numpy(rng.integers(0, 256, size=(n_pages, unit), dtype=np.uint8)).pin_memory()
+    table = rng.permutation(n_pages)[: cfg.batch * nb].astype(np.int32).reshape(cfg.batch, nb)
+    pool0 = rng.integers(0, 256, size=(cfg.batch, C, unit), dtype=np.uint8)
+    pool = torch.from_numpy(pool0).cuda()
+    cap = 8
+    lists = np.zeros((cfg.batch, cap, 4), np.int32)
+    counts = np.zeros(cfg.batch, np.int32)
+    pairs_of = []
+    for s in range(cfg.batch):
+        # extents of 1..3 logical blocks; destination slots consecutive inside an extent
+        src = [(1, 2), (7, 1), (20, 3)][: s + 1]
+        dst, before, pairs = 0, 0, []
+        for i, (b0, n) in enumerate(src):
+            lists[s, i] = (b0, dst, n, before)
+            pairs += [(b0 + k, dst + k) for k in range(n)]
+            dst += n + 1
+            before += n
+        counts[s] = len(src)
+        pairs_of.append(np.asarray(pairs, np.int32))
+    pi.recall_gather_scatter(0, arena, pool, torch.from_numpy(lists).cuda(), torch.from_numpy(counts).cuda(),
+                             page_table=torch.from_numpy(table).cuda(), n_pages=n_pages)
+    torch.cuda.synchronize()
+    assert pi.status()[0] == 0
+    got = pool.cpu().numpy()
+    for s in range(cfg.batch):
+        ref = pool0[s].copy()
+        oracle.recall_paged(arena.numpy(), table[s], ref, pairs_of[s], unit)
+        assert np.array_equal(got[s], ref)
+    # a page index outside the arena is reported, not followed
+    bad = table.copy()
+    bad[0, 1] = n_pages
+    pi.recall_gather_scatter(0, arena, pool, torch.from_numpy(lists).cuda(), torch.from_numpy(counts).cuda(),
+                             page_table=torch.from_numpy(bad).cuda(), n_pages=n_pages)
+    torch.cuda.synchronize()
+    st = pi.status()
+    assert st[0] == -8 and st[1] == 3, st
+    pi.close()
+
+
+def test_pipelined_session_on_a_paged_host_store_with_append():
+    """The whole decode step, two layers, pipelined, blocks scattered over a paged arena, one token
+    appended per step: every stage against the oracle, and the host store after the appends."""
+    from tests.parity import run_session_sampled
+    cfg = tiny_config(batch=4, ctx=4096, n_q_heads=32, n_kv_heads=8, budget_blocks=40, resident_frac=0.3, n_layers=2)
+    stats = run_session_sampled(cfg, steps=10, sample_seqs=[1, 2], append=True, ctx_start=4096 - 18, paged=True)
+    assert stats["misses"] > 0
