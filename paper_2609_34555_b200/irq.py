@@ -305,7 +305,7 @@ if __name__ == "__main__":
     ap.add_argument("--offload-layers", type=int, default=256)
     ap.add_argument("--normal-batch", type=int, default=64)
     ap.add_argument("--normal-ctx", type=int, default=4096)
-    ap.add_argument("--recall-ctas", type=int, default=0)
+    ap.add_argument("--recall-ctas", type=int, default=10, help="one recall launch at a time here: 10 CTAs (the library default of 5 is sized for two launches side by side)")
     a = ap.parse_args()
     for r in run_on_gpu(a.offload_layers, a.normal_batch, a.normal_ctx, recall_ctas=a.recall_ctas):
         print(json.dumps(r))

@@ -48,6 +48,8 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--reps", type=int, default=8)
     ap.add_argument("--out", default="")
+    ap.add_argument("--recall-ctas", type=int, default=10,
+                    help="CTAs of the one launch timed here (the library default of 5 is sized for two launches side by side)")
     ap.add_argument("--blocks", default="16,32,64")
     ap.add_argument("--misses", default="8,32,128,512,2048")
     args = ap.parse_args()
@@ -56,7 +58,7 @@ def main():
     for B in [int(x) for x in args.blocks.split(",")]:
         cfg = get_config("c5").replace(block_tokens=B, budget_blocks=max(128 * 16 // B, 16))
         nb, C, Hkv = cfg.n_blocks, cfg.pool_slots, cfg.n_kv_heads
-        pi = PulseInfer.from_workload(cfg)
+        pi = PulseInfer.from_workload(cfg, recall_ctas=args.recall_ctas)
         host = torch.empty((cfg.batch, nb, cfg.block_bytes // 2), dtype=torch.bfloat16, pin_memory=True)
         host.view(torch.int16).random_(0, 30000)
         buf = LayerBuffers(pi, cfg.batch, dev)
