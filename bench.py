@@ -186,11 +186,11 @@ def run_ours(args) -> dict:
     t_setup = time.time()
     n_e2e = K if not args.no_e2e else 0
     n_serial = min(K, 4)
-    total_steps = args.settle + W + K + n_serial + n_e2e
+    total_steps = args.settle + W + K + 2 * n_serial + n_e2e
     pi, sess, R = build_session(cfg, rank, args.host_layers, world, args.recall_ctas,
                                 ctx_start=cfg.ctx - total_steps - 1 if args.append else 0, paged=args.paged,
                                 recall_streams=args.recall_streams)
-    q_all = make_all_queries(cfg, args.settle + W + K + n_serial + n_e2e, dev)
+    q_all = make_all_queries(cfg, total_steps, dev)
     setup_s = time.time() - t_setup
 
     # pinned host -> device copy peak, measured in this run (1 GiB, best of 10)
@@ -245,7 +245,9 @@ def run_ours(args) -> dict:
     # ---------------- timed region: K pipelined decode steps, inputs resident in HBM
     sampler = ClockSampler(local)
     sampler.start()
-    timer = StageTimer()
+    # the stage times of this region come from the events that order the streams anyway (no event
+    # is added to any stream: extra events on the recall streams cost about 6 % of the rate)
+    timer = StageTimer(light=True)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
@@ -256,10 +258,18 @@ def run_ours(args) -> dict:
     clocks = sampler.stop()
     ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
     stats = pi.stats(reset=True)
-    stages = timer.summary()
+    stages = timer.light_summary(e0)
     status = pi.status()
     if status[0] != 0:
         raise RuntimeError(f"device status after the timed region: {status}")
+
+    # ---------------- the same pipelined form with events around every call (per-call picture)
+    det_timer = StageTimer()
+    for _ in range(n_serial):
+        sess.decode_step(q_all[t], timer=det_timer, resident_script=script(t), new_kv=new_kv); t += 1
+    torch.cuda.synchronize()
+    det = det_timer.summary()
+    pi.stats(reset=True)
 
     # ---------------- serial form (one stream), a few steps, for the per-stage picture
     ser_timer = StageTimer()
@@ -277,20 +287,20 @@ def run_ours(args) -> dict:
     e2e = None
     if n_e2e:
         q_host = q_all[t:t + n_e2e].cpu().pin_memory()
-        out_host = torch.empty(sess.out.shape, dtype=torch.bfloat16, pin_memory=True)
-        q_dev = torch.empty_like(q_all[0])
+        out_host = [torch.empty(sess.out.shape, dtype=torch.bfloat16, pin_memory=True) for _ in range(2)]
         barrier()
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a0.record()
-        t_e2e = t
-        for i in range(n_e2e):
-            sess.decode_step_from_host(q_host[i], out_host, q_dev, resident_script=script(t_e2e + i))
+        # every step: its queries come up from pinned host memory and its outputs go back to pinned host
+        # memory; both copies are double-buffered so that they run beside the neighbouring steps
+        sess.decode_steps_from_host([q_host[i] for i in range(n_e2e)], out_host,
+                                    resident_scripts=None if scripts is None else [script(t + i) for i in range(n_e2e)])
         a1.record()
         barrier()
         e2e_ms = max_over_ranks(a0.elapsed_time(a1), world, dev)
         e2e_stats = pi.stats(reset=True)
         e2e = dict(value=whole_job_value(world, n_e2e, cfg.n_layers, e2e_ms), unit="layer-steps/s",
-                   h2d_bytes_per_step=int(q_dev.numel() * 2), d2h_bytes_per_step=int(out_host.numel() * 2),
+                   h2d_bytes_per_step=int(q_host[0].numel() * 2), d2h_bytes_per_step=int(out_host[0].numel() * 2),
                    misses_per_seq_layer_step=e2e_stats["missing_blocks"] / max(1, e2e_stats["sequences"]),
                    note="host KV store is read by the recall kernel in both forms")
 
@@ -298,7 +308,11 @@ def run_ours(args) -> dict:
     traffic = NCU_DRAM_TRAFFIC.get(base.name, {}) if args.layers == 0 else {}
     n_launch = K * cfg.n_layers
     recall_bytes = stats["missing_blocks"] * cfg.block_bytes
-    recall_s = timer.busy_ms("recall", e0) * 1e-3        # union of the launches' intervals: they overlap across streams
+    # union of the launches' intervals (they overlap across the recall streams); the first launch of
+    # each recall stream has no bounded start and is left out of bytes and time alike
+    n_rec = stages["recall"]["launches"]
+    recall_bytes = recall_bytes * n_rec / max(1, n_launch)
+    recall_s = stages["recall"]["busy_ms"] * 1e-3
     attn_bytes_launch = stats["selected_blocks"] / max(1, n_launch) * cfg.block_bytes + 2 * cfg.batch * cfg.n_q_heads * 128 * 2
     score_bytes_launch = cfg.batch * cfg.n_blocks * 512 + cfg.batch * cfg.group * 128 * 2
     def hbm_entry(name, bytes_launch, st, traffic):
@@ -328,18 +342,19 @@ def run_ours(args) -> dict:
         "roofline": {"kernel": "recall_kernel", "bound": "host_link_h2d", "achieved": recall_gbs, "peak": h2d_gbs,
                      "unit": "GB/s", "frac": recall_gbs / h2d_gbs,
                      "peak_source": "pinned cudaMemcpyAsync H2D of 1 GiB, best of 10, this run (nominal 64 GB/s PCIe Gen5 x16)",
-                     "traffic": None, "bytes_per_launch": int(recall_bytes / max(1, n_launch)),
-                     "mean_us": stages["recall"]["mean_ms"] * 1e3, "busy_us_per_launch": recall_s * 1e6 / max(1, n_launch),
+                     "traffic": None, "bytes_per_launch": int(recall_bytes / max(1, n_rec)),
+                     "mean_us": stages["recall"]["mean_ms"] * 1e3, "busy_us_per_launch": recall_s * 1e6 / max(1, n_rec),
                      "concurrent_streams": len(sess.recall_streams),
                      "achieved_is": "recalled bytes / time during which a recall launch was running (launches of consecutive "
                                     "layers overlap across the recall streams; with one stream this is bytes per launch / "
                                     "mean launch duration)",
                      "alone": {"achieved": ser_recall_gbs, "frac": ser_recall_gbs / h2d_gbs}},
-        "rooflines": [hbm_entry("attn_kernel + attn_merge_kernel (pipelined region, recall running beside it)", attn_bytes_launch, stages["attn"], traffic.get("attn_kernel")),
-                      hbm_entry("score_select_kernel (pipelined region)", score_bytes_launch, stages["score_select"], traffic.get("score_select_kernel")),
+        "rooflines": [hbm_entry("attn_kernel + attn_merge_kernel (timed region, recalls running beside it)", attn_bytes_launch, stages["attn"], traffic.get("attn_kernel")),
+                      hbm_entry("score_select_kernel (pipelined form, events around every call)", score_bytes_launch, det["score_select"], traffic.get("score_select_kernel")),
                       hbm_entry("attn_kernel + attn_merge_kernel (serial form, nothing else running)", attn_bytes_launch, ser["attn"], traffic.get("attn_kernel")),
                       hbm_entry("score_select_kernel (serial form)", score_bytes_launch, ser["score_select"], traffic.get("score_select_kernel"))],
         "stages_us": {k: v["mean_ms"] * 1e3 for k, v in stages.items() if v["launches"]},
+        "stages_us_events_around_every_call": {k: v["mean_ms"] * 1e3 for k, v in det.items() if v["launches"]},
         "serial": {"layer_steps_per_s": cfg.n_layers / (serial_ms * 1e-3),
                    "stages_us": {k: v["mean_ms"] * 1e3 for k, v in ser.items() if v["launches"]}},
         "h2d_peak_gbs": h2d_gbs,

@@ -98,13 +98,59 @@ class RecallPath:
 
 
 class StageTimer:
-    """CUDA events around each call of a decode step, on the stream the call runs on."""
+    """CUDA events around each call of a decode step, on the stream the call runs on.
+
+    `light=True` adds no event to any stream: the events the pipelined step records anyway to
+    order its streams (selection+diff done, recall landed, attention done) are created with
+    timing enabled and kept, and the stage intervals are reconstructed from their timestamps
+    afterwards (`light_summary`).  Extra events between the kernels of the recall streams cost
+    the pipelined step about 6 % of its rate, which is why the timed region uses this form."""
 
     STAGES = ("append", "score_select", "diff", "recall", "attn")
 
-    def __init__(self, stages=None):
+    def __init__(self, stages=None, light: bool = False):
         self.stages = tuple(stages) if stages else self.STAGES
         self.pairs = {s: [] for s in self.stages}
+        self.light = light
+        self.records = []          # light form: (layer, recall stream index, ev_diff, ev_recall, ev_attn) in launch order
+
+    def sync_events(self, layer: int, recall_stream: int):
+        evs = tuple(torch.cuda.Event(enable_timing=True) for _ in range(3))
+        self.records.append((layer, recall_stream) + evs)
+        return evs
+
+    def light_summary(self, base: torch.cuda.Event) -> dict:
+        """Stage intervals of the light form on the clock of `base` (a timing event recorded before
+        the first step; call after a synchronize).  A stage starts when its stream is free and its
+        input event has fired: recall = max(diff done, previous recall of the same stream done) ->
+        recall landed; attention = max(recall landed, previous attention done) -> attention done;
+        select+diff = max(previous diff done, this layer's previous attention done) -> diff done.
+        The first launch of each stream (no predecessor to bound its start) is left out."""
+        last_recall, last_attn_of_layer = {}, {}
+        prev_diff = prev_attn = None
+        spans = {"recall": [], "attn": [], "select_diff": []}
+        for layer, rs, evd, evr, eva in self.records:
+            td, tr, ta = base.elapsed_time(evd), base.elapsed_time(evr), base.elapsed_time(eva)
+            if rs in last_recall:
+                spans["recall"].append((max(td, last_recall[rs]), tr))
+            if prev_attn is not None:
+                spans["attn"].append((max(tr, prev_attn), ta))
+            if prev_diff is not None:
+                spans["select_diff"].append((max(prev_diff, last_attn_of_layer.get(layer, 0.0)), td))
+            last_recall[rs], last_attn_of_layer[layer] = tr, ta
+            prev_diff, prev_attn = td, ta
+        out = {}
+        for name, lst in spans.items():
+            ms = [b - a for a, b in lst]
+            busy, end = 0.0, float("-inf")
+            for a, b in sorted(lst):
+                if a > end:
+                    busy, end = busy + (b - a), b
+                elif b > end:
+                    busy, end = busy + (b - end), b
+            out[name] = dict(launches=len(ms), total_ms=float(sum(ms)), mean_ms=float(sum(ms) / max(1, len(ms))),
+                             busy_ms=float(busy))
+        return out
 
     def wants(self, stage: str) -> bool:
         return stage in self.pairs
@@ -223,18 +269,20 @@ class DecodeSession:
                                  kv_for_digest=kv_dev, page_table=pt)
 
     def decode_step(self, q: torch.Tensor, overlapped: bool = True, timer: Optional[StageTimer] = None,
-                    resident_script: Optional[torch.Tensor] = None, new_kv=None) -> torch.Tensor:
-        """q: device bf16 [n_layers][batch][Hq][D].  Returns self.out ([n_layers][batch][Hq][D]);
+                    resident_script: Optional[torch.Tensor] = None, new_kv=None,
+                    out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """q: device bf16 [n_layers][batch][Hq][D].  Returns `out` (default self.out, [n_layers][batch][Hq][D]);
         valid once the current stream has caught up.  resident_script (int32 [n_layers][batch][C]):
         workloads with scripted miss counts reset each layer's tables to these hot-set contents
         before the layer's diff (pool contents are not refreshed: timing runs only).
         new_kv = (k_new, v_new), each bf16 [n_layers][batch][Hkv][D]: the step's new token is appended
         to every layer first (pool slot, host store, digest) and the context grows by one.
 
-        Overlapped form: three streams.  Selection and diff of every layer run ahead on one
-        stream, the recall pulls follow on a second one (the host link stays busy back to
-        back), and each layer's attention runs on the current stream once its recall landed."""
+        Overlapped form: selection and diff of every layer run ahead on one stream, the recall
+        pulls follow on the recall streams in rotation (the host link stays busy back to back),
+        and each layer's attention runs on the current stream once its recall landed."""
         pi = self.pi
+        out = self.out if out is None else out
         self.step_count += 1
         step = self.step_count
         main = torch.cuda.current_stream(self.device)
@@ -248,10 +296,19 @@ class DecodeSession:
                 self.ctx_len += 1
         for l in range(self.n_layers):
             b, host, pt = self.bufs[l], self.host_region(l), self.page_table(l)
-            rec_s = self.recall_streams[l % len(self.recall_streams)] if overlapped else main
+            rs_i = l % len(self.recall_streams)
+            rec_s = self.recall_streams[rs_i] if overlapped else main
+            tm = timer
+            if overlapped and tm is not None and tm.light:
+                # the ordering events double as timestamps: no extra work on any stream
+                self._ev_diff[l], self._ev_recall[l], ev_attn_new = tm.sync_events(l, rs_i)
+                tm = None
+            else:
+                ev_attn_new = None
             if overlapped and step > 1:
                 sel_s.wait_event(self._ev_attn[l])         # last step's attention still reads this layer's lists and pool
-            tm = timer
+            if ev_attn_new is not None:
+                self._ev_attn[l] = ev_attn_new
             if resident_script is not None:
                 pi.table_init(resident_script[l], b.block_table, b.slot_block, b.slot_stamp, stream=sel_s)
             if new_kv is not None:
@@ -277,7 +334,7 @@ class DecodeSession:
                 main.wait_event(self._ev_recall[l])
             t4 = tm.mark(main) if tm and tm.wants("attn") else None
             pi.sparse_decode_attn(l, q[l], b.pool, b.sel_slots, b.sel_blocks, b.sel_count, self.ctx_len,
-                                  self.out[l], None, stream=main)
+                                  out[l], None, stream=main)
             t5 = tm.mark(main) if tm and tm.wants("attn") else None
             if overlapped:
                 self._ev_attn[l].record(main)
@@ -286,7 +343,52 @@ class DecodeSession:
                 if t2 is not None: tm.add("diff", t1, t2)
                 if t2r is not None: tm.add("recall", t2r, t3)
                 if t4 is not None: tm.add("attn", t4, t5)
-        return self.out
+        return out
+
+    def decode_steps_from_host(self, q_hosts, out_hosts, resident_scripts=None) -> None:
+        """End-to-end form over several steps with the copies off the critical path: step i's queries
+        (pinned host, [n_layers][batch][Hq][D]) are uploaded on a copy stream while step i-1 computes,
+        step i's outputs are downloaded to out_hosts[i % len(out_hosts)] (pinned host) while step i+1
+        computes.  Queries and outputs are double-buffered on the device.  Returns once everything is
+        enqueued; out_hosts are valid after a synchronize."""
+        main = torch.cuda.current_stream(self.device)
+        if not hasattr(self, "_copy_s"):
+            self._copy_s = torch.cuda.Stream(self.device)
+            self._q2 = [torch.empty(self.out.shape, dtype=torch.bfloat16, device=self.device) for _ in range(2)]
+            self._out2 = [torch.empty_like(self.out) for _ in range(2)]
+        cp = self._copy_s
+        n = len(q_hosts)
+        ev_up = [torch.cuda.Event() for _ in range(n)]
+        ev_done = [torch.cuda.Event() for _ in range(n)]
+        ev_down = [torch.cuda.Event() for _ in range(n)]
+        start = torch.cuda.Event()
+        start.record(main)
+        cp.wait_event(start)
+
+        def upload(i):
+            with torch.cuda.stream(cp):
+                if i >= 2:
+                    cp.wait_event(ev_done[i - 2])            # the step that last read this query buffer
+                self._q2[i % 2].copy_(q_hosts[i], non_blocking=True)
+                ev_up[i].record(cp)
+
+        upload(0)
+        for i in range(n):
+            if i + 1 < n:
+                upload(i + 1)
+            main.wait_event(ev_up[i])
+            if i >= 2:
+                main.wait_event(ev_down[i - 2])              # the download that last read this output buffer
+            self.decode_step(self._q2[i % 2], overlapped=True, out=self._out2[i % 2],
+                             resident_script=None if resident_scripts is None else resident_scripts[i])
+            ev_done[i].record(main)
+            with torch.cuda.stream(cp):
+                cp.wait_event(ev_done[i])
+                out_hosts[i % len(out_hosts)].copy_(self._out2[i % 2], non_blocking=True)
+                ev_down[i].record(cp)
+        main.wait_event(ev_down[n - 1])
+        if n >= 2:
+            main.wait_event(ev_down[n - 2])
 
     def decode_step_from_host(self, q_host: torch.Tensor, out_host: torch.Tensor, q_dev: torch.Tensor,
                               resident_script: Optional[torch.Tensor] = None) -> None:

@@ -389,3 +389,41 @@ def test_pipelined_session_on_a_paged_host_store_with_append():
     cfg = tiny_config(batch=4, ctx=4096, n_q_heads=32, n_kv_heads=8, budget_blocks=40, resident_frac=0.3, n_layers=2)
     stats = run_session_sampled(cfg, steps=10, sample_seqs=[1, 2], append=True, ctx_start=4096 - 18, paged=True)
     assert stats["misses"] > 0
+
+
+def test_double_buffered_host_stepping_matches_plain_stepping():
+    """decode_steps_from_host (queries uploaded and outputs downloaded beside the neighbouring steps)
+    must return, step by step, exactly what decode_step returns from the same state."""
+    import numpy as np
+    import torch
+    from paper_2609_34555_b200 import PulseInfer
+    from paper_2609_34555_b200.runner import DecodeSession
+    from workloads import generate as gen
+    cfg = tiny_config(batch=3, ctx=2048, n_q_heads=16, n_kv_heads=4, budget_blocks=24, resident_frac=0.3, n_layers=3)
+    steps = 5
+    outs = []
+    for form in ("plain", "host"):
+        pi = PulseInfer.from_workload(cfg)
+        sess = DecodeSession(pi, cfg.batch, cfg.n_layers)
+        sess.ctx_len.fill_(cfg.ctx)
+        for l in range(cfg.n_layers):
+            kv = gen.make_kv(cfg, l, device=sess.device)
+            sess.load_layer(l, kv, torch.from_numpy(gen.initial_resident(cfg, l)).to(sess.device))
+        q_all = torch.stack([gen.make_queries(cfg, l, steps, device=sess.device) for l in range(cfg.n_layers)], 1).contiguous()
+        if form == "plain":
+            got = []
+            for t in range(steps):
+                sess.decode_step(q_all[t])
+                torch.cuda.synchronize()
+                got.append(sess.out.cpu().clone())
+        else:
+            q_host = q_all.cpu().pin_memory()
+            out_host = [torch.empty(sess.out.shape, dtype=torch.bfloat16, pin_memory=True) for _ in range(steps)]
+            sess.decode_steps_from_host([q_host[t] for t in range(steps)], out_host)
+            torch.cuda.synchronize()
+            got = [o.clone() for o in out_host]
+        assert pi.status()[0] == 0
+        outs.append(got)
+        pi.close()
+    for t in range(steps):
+        assert torch.equal(outs[0][t].view(torch.int16), outs[1][t].view(torch.int16)), f"step {t}"
