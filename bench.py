@@ -164,6 +164,39 @@ def whole_job_value(world: int, steps: int, n_layers: int, ms: float) -> float:
     return world * steps * n_layers / (ms * 1e-3)
 
 
+def parse_cpulist(text: str) -> set:
+    """'0-3,8,10-11' -> {0, 1, 2, 3, 8, 10, 11} (the format of sysfs cpulist files)."""
+    cpus = set()
+    for part in text.strip().split(","):
+        if not part:
+            continue
+        lo, _, hi = part.partition("-")
+        cpus.update(range(int(lo), int(hi or lo) + 1))
+    return cpus
+
+
+def bind_near_gpu(index: int):
+    """Multi-rank runs: keep this process (and so the pages of the pinned host store it is about to
+    allocate, which land on the node of the allocating thread) on the NUMA node of its GPU, so that
+    every rank's recall crosses only its own GPU's host link.  Best effort: returns the node or None."""
+    try:
+        bus = torch.cuda.get_device_properties(index).pci_bus_id
+        dom = torch.cuda.get_device_properties(index).pci_domain_id
+        dev_id = torch.cuda.get_device_properties(index).pci_device_id
+        path = Path(f"/sys/bus/pci/devices/{dom:04x}:{bus:02x}:{dev_id:02x}.0/numa_node")
+        node = int(path.read_text().strip())
+        if node < 0:
+            return None
+        cpus = parse_cpulist(Path(f"/sys/devices/system/node/node{node}/cpulist").read_text())
+        cpus &= os.sched_getaffinity(0)
+        if not cpus:
+            return None
+        os.sched_setaffinity(0, cpus)
+        return node
+    except Exception:                                # noqa: BLE001 - placement hint only
+        return None
+
+
 def run_ours(args) -> dict:
     from paper_2609_34555_b200 import h2d_copy_ms
     from paper_2609_34555_b200.runner import StageTimer
@@ -174,9 +207,11 @@ def run_ours(args) -> dict:
     world = int(os.environ.get("WORLD_SIZE", "1"))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
+    numa_node = None
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
+        numa_node = bind_near_gpu(local)
     base = get_config(args.config)
     cfg = rank_config(base, rank)
     if args.layers > 0:                       # profiling only: fewer layers of the same shape
@@ -359,6 +394,7 @@ def run_ours(args) -> dict:
                                f"Hq/Hkv {cfg.n_q_heads}/{cfg.n_kv_heads}, block {cfg.block_tokens}, budget {cfg.budget_blocks} "
                                f"blocks, pool {cfg.pool_slots} slots/seq/layer, AR(1) queries a={cfg.ar1}",
                    "host_layout": "paged arena, random page order" if args.paged else "block-major per sequence",
+                   "numa_node_of_rank0": numa_node,
                    "host_kv_layers": R, "host_kv_pinned_gb": R * cfg.batch * cfg.n_blocks * cfg.block_bytes / 2 ** 30,
                    "l2": f"inputs larger than L2 (pool reads {cfg.batch * cfg.budget_blocks * cfg.block_bytes / 2**20:.0f} MiB and digests "
                          f"{cfg.batch * cfg.n_blocks * 512 / 2**20:.0f} MiB per layer-step, {cfg.n_layers} distinct layers)",

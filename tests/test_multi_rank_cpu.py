@@ -55,3 +55,13 @@ def test_two_ranks_shard_sequences_and_take_the_max_time():
     assert seed0 != seed1 and sigs0 == sigs1 and sigs0[0] != sigs0[1]
     assert ms0 == ms1 == 20.0                        # the slower rank's time, on both
     assert v0 == v1 == 2 * 4 * 1 / 20e-3             # both ranks' layer-steps over the max time
+
+
+def test_cpulist_parser_and_numa_binding_falls_back_quietly():
+    sys.path.insert(0, str(ROOT))
+    import bench
+    assert bench.parse_cpulist("0-3,8,10-11\n") == {0, 1, 2, 3, 8, 10, 11}
+    assert bench.parse_cpulist("5") == {5} and bench.parse_cpulist("") == set()
+    before = os.sched_getaffinity(0)
+    assert bench.bind_near_gpu(0) is None            # no GPU here: a placement hint must never raise
+    assert os.sched_getaffinity(0) == before
