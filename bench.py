@@ -6,7 +6,8 @@
 One "step" is one decode step of the whole batch: every layer runs one layer-step of the
 path.  The metric is layer-steps per second.  Rank 0 prints ONE JSON line.
 
-  value        inputs (queries) already in HBM, the pipelined three-stream form
+  value        inputs (queries) already in HBM, the pipelined form (selection stream, two recall
+               streams, attention stream)
   e2e          the same through DecodeSession with the queries coming from pinned host memory
                and the outputs copied back to pinned host memory inside the timed region
   roofline     the kernel that dominates the step (the recall pull, bound by the host link)
