@@ -37,7 +37,9 @@ import torch
 METRIC = "decode layer-steps/s (select+recall+attn); recall GB/s vs measured H2D peak"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (attn_kernel_c2.txt, score_select_kernel_c2.txt): same per-layer shapes as the bench
-NCU_DRAM_TRAFFIC = {"c2": {"attn_kernel": 134.5e6 + 4.3e6, "score_select_kernel": 18.9e6}}
+# (recall_kernel: its reads cross the host link and its 5 MB of writes stay in L2 during the launch,
+# so DRAM sees next to nothing)
+NCU_DRAM_TRAFFIC = {"c2": {"attn_kernel": 134.5e6 + 4.3e6, "score_select_kernel": 18.9e6, "recall_kernel": 21.0e3}}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -408,7 +410,9 @@ def run_ours(args) -> dict:
         "roofline": {"kernel": "recall_kernel", "bound": "host_link_h2d", "achieved": recall_gbs, "peak": h2d_gbs,
                      "unit": "GB/s", "frac": recall_gbs / h2d_gbs,
                      "peak_source": "pinned cudaMemcpyAsync H2D of 1 GiB, best of 10, this run (nominal 64 GB/s PCIe Gen5 x16)",
-                     "traffic": None, "bytes_per_launch": int(recall_bytes / max(1, n_rec)),
+                     "traffic": traffic.get("recall_kernel"),
+                     "traffic_note": "DRAM bytes per launch under ncu: the reads come over the host link, the writes stay in L2",
+                     "bytes_per_launch": int(recall_bytes / max(1, n_rec)),
                      "mean_us": stages["recall"]["mean_ms"] * 1e3, "busy_us_per_launch": recall_s * 1e6 / max(1, n_rec),
                      "concurrent_streams": len(sess.recall_streams),
                      "achieved_is": "recalled bytes / time during which a recall launch was running (launches of consecutive "
