@@ -546,7 +546,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="cut the layer stack (for profiler captures only)")
     ap.add_argument("--recall-ctas", type=int, default=0, help="CTAs of the recall kernel (0 = library default)")
     ap.add_argument("--append", action="store_true", help="grow the context: append one synthetic token per step and layer")
-    ap.add_argument("--attn-ctas", type=int, default=0, help="CTAs of the attention kernel (0 = one per SM)")
+    ap.add_argument("--attn-ctas", type=int, default=0, help="CTAs of the attention kernel (0 = library default)")
     ap.add_argument("--recall-streams", type=int, default=2, help="streams the recall launches rotate over")
     ap.add_argument("--paged", action="store_true", help="host store as an arena of pages in random order behind a page table")
     ap.add_argument("--no-e2e", action="store_true")

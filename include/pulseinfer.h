@@ -57,7 +57,7 @@ typedef struct {
     int32_t pool_slots;                       /* C per (seq, layer); C >= K                       */
     int32_t max_batch, max_blocks;            /* capacities: batch <= max_batch, NB = max_blocks  */
     int32_t recall_ctas;                      /* CTAs per recall launch, 0 = default (5)           */
-    int32_t attn_ctas;                        /* CTAs of the attention kernel, 0 = one per SM     */
+    int32_t attn_ctas;                        /* CTAs of the attention kernel, 0 = default (#SMs - 20) */
     const int32_t* solo_head;                 /* host [n_layers]: retrieval KV head per layer (copied) */
 } pi_config;
 

@@ -56,7 +56,9 @@ extern "C" int pi_create(const pi_config* cfg, pi_ctx** out) {
     if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, c->device);
     if (e != cudaSuccess) { (void)cudaGetLastError(); pi_destroy(c); return PI_ERR_CUDA; }
     c->n_sms = prop.multiProcessorCount;
-    c->attn_ctas = cfg->attn_ctas > 0 ? cfg->attn_ctas : c->n_sms;
+    // the persistent attention grid saturates HBM from about 80 SMs on; leaving 20 SMs to the kernels
+    // of the other streams (recall CTAs, score/select, diff) costs it nothing and keeps them off its SMs
+    c->attn_ctas = cfg->attn_ctas > 0 ? cfg->attn_ctas : (c->n_sms > 40 ? c->n_sms - 20 : c->n_sms);
     // five CTAs per launch (40 warps x 4 KB in flight): two launches running side by side on two
     // streams saturate the host link of a B200 and cover each other's fixed costs; one launch alone
     // still reaches 0.97 of what ten CTAs do, and more requests in flight only queue up
