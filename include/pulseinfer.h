@@ -188,6 +188,18 @@ int pi_sparse_decode_attn(pi_ctx* ctx, int layer, int batch, const void* q_dev, 
                           const int32_t* sel_count_dev, const int32_t* ctx_len_dev, void* out_dev,
                           float* lse_dev, void* stream);
 
+/* The same attention when every KV head carries its own selection (the headwise strategy of the
+ * paper's selection study, Sec. 4.4.1, as produced by pi_score_select_strategy(PI_SELECT_HEADWISE) +
+ * pi_diff_misses over batch*Hkv rows + per-head fragment recall): query heads of KV head h attend
+ * over the blocks of list (s, h) only, whose K/V fragments sit in the pool at
+ * [slot][h] (the pool keeps the [batch][C][Hkv][2][B][D] layout; slots are per head).
+ *   sel_slots_dev / sel_blocks_dev [batch][Hkv][K]; sel_count_dev [batch][Hkv]; the rest as above.
+ * Heads of one sequence may select different numbers of blocks. */
+int pi_sparse_decode_attn_headwise(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* pool_dev,
+                                   const int32_t* sel_slots_dev, const int32_t* sel_blocks_dev,
+                                   const int32_t* sel_count_dev, const int32_t* ctx_len_dev, void* out_dev,
+                                   float* lse_dev, void* stream);
+
 /* The step before the path: the decode step's new token joins the cache.  (The paper implies it:
  * an offloaded request keeps its full KV in CPU memory and its sink, local and hot middle tokens
  * on the GPU, Sec. 4.2 and Sec. 5 Setup; it does not describe the operation.)  For every sequence

@@ -23,7 +23,7 @@ ERR_NAMES = {
 EXTENT_DTYPE = torch.int32      # a pi_extent is four int32: src_unit, dst_unit, n_units, units_before
 
 EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_score_select_noalloc", "pi_score_select_strategy", "pi_diff_misses", "pi_recall_gather_scatter",
-           "pi_recall_gather_scatter_paged", "pi_sparse_decode_attn", "pi_append_kv", "pi_append_kv_paged", "pi_build_digests", "pi_build_digests_all", "pi_table_init", "pi_h2d_copy_ms",
+           "pi_recall_gather_scatter_paged", "pi_sparse_decode_attn", "pi_sparse_decode_attn_headwise", "pi_append_kv", "pi_append_kv_paged", "pi_build_digests", "pi_build_digests_all", "pi_table_init", "pi_h2d_copy_ms",
            "pi_get_status", "pi_get_stats", "pi_clear_status", "pi_strerror"]
 
 
@@ -67,6 +67,7 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.pi_score_select_strategy.argtypes = [c_void_p, c_int, c_int, c_int, vp, vp, i32p, i32p, i32p, vp, vp]
     lib.pi_build_digests_all.argtypes = [c_void_p, c_int, vp, c_int64, i32p, vp, vp]
     lib.pi_sparse_decode_attn.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, i32p, vp, vp, vp]
+    lib.pi_sparse_decode_attn_headwise.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, i32p, vp, vp, vp]
     lib.pi_append_kv.argtypes = [c_void_p, c_int, c_int, c_uint32, vp, vp, i32p, vp, c_int64, vp, i32p, i32p, u32p, vp, vp]
     lib.pi_build_digests.argtypes = [c_void_p, c_int, c_int, vp, c_int64, i32p, vp, vp]
     lib.pi_table_init.argtypes = [c_void_p, c_int, i32p, i32p, i32p, u32p, vp]
@@ -233,11 +234,14 @@ class PulseInfer:
             unit_bytes or self.block_bytes, unit_stride, list_offset, _stream(stream)))
 
     def sparse_decode_attn(self, layer: int, q, pool, sel_slots, sel_blocks, sel_count, ctx_len, out, lse=None,
-                           stream=None) -> None:
+                           stream=None, headwise: bool = False) -> None:
+        """headwise=True: sel_slots / sel_blocks are [batch][Hkv][K] (or [batch*Hkv][K]) and sel_count
+        [batch][Hkv]: every KV head attends over its own selection."""
         batch = q.shape[0]
         if not pool.is_cuda or not pool.is_contiguous():
             raise TypeError("pool: expected a contiguous CUDA tensor")
-        _check("pi_sparse_decode_attn", self._lib.pi_sparse_decode_attn(
+        fn = self._lib.pi_sparse_decode_attn_headwise if headwise else self._lib.pi_sparse_decode_attn
+        _check("pi_sparse_decode_attn_headwise" if headwise else "pi_sparse_decode_attn", fn(
             self._ctx, layer, batch, _dev(q, torch.bfloat16, "q"), pool.data_ptr(),
             _dev(sel_slots, torch.int32, "sel_slots"), _dev(sel_blocks, torch.int32, "sel_blocks"),
             _dev(sel_count, torch.int32, "sel_count"), _dev(ctx_len, torch.int32, "ctx_len"),

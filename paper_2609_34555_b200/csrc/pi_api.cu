@@ -216,10 +216,9 @@ extern "C" int pi_recall_gather_scatter_paged(pi_ctx* ctx, int layer, int n_list
                        unit_bytes, unit_stride_bytes, list_offset_bytes, stream);
 }
 
-extern "C" int pi_sparse_decode_attn(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* pool_dev,
-                                     const int32_t* sel_slots_dev, const int32_t* sel_blocks_dev,
-                                     const int32_t* sel_count_dev, const int32_t* ctx_len_dev, void* out_dev,
-                                     float* lse_dev, void* stream) {
+static int attn_call(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* pool_dev,
+                     const int32_t* sel_slots_dev, const int32_t* sel_blocks_dev, const int32_t* sel_count_dev,
+                     const int32_t* ctx_len_dev, void* out_dev, float* lse_dev, int headwise, void* stream) {
     int rc = check_call(ctx, layer, batch);
     if (rc != PI_OK) return rc;
     if (!q_dev || !pool_dev || !sel_slots_dev || !sel_blocks_dev || !sel_count_dev || !ctx_len_dev || !out_dev)
@@ -227,7 +226,24 @@ extern "C" int pi_sparse_decode_attn(pi_ctx* ctx, int layer, int batch, const vo
     if (!pi_aligned16(q_dev) || !pi_aligned16(out_dev) || (reinterpret_cast<uintptr_t>(pool_dev) & 127u))
         return PI_ERR_BAD_ALIGN;
     return pi_launch_attn(ctx, batch, q_dev, pool_dev, sel_slots_dev, sel_blocks_dev, sel_count_dev,
-                          ctx_len_dev, out_dev, lse_dev, static_cast<cudaStream_t>(stream));
+                          ctx_len_dev, out_dev, lse_dev, headwise, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int pi_sparse_decode_attn(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* pool_dev,
+                                     const int32_t* sel_slots_dev, const int32_t* sel_blocks_dev,
+                                     const int32_t* sel_count_dev, const int32_t* ctx_len_dev, void* out_dev,
+                                     float* lse_dev, void* stream) {
+    return attn_call(ctx, layer, batch, q_dev, pool_dev, sel_slots_dev, sel_blocks_dev, sel_count_dev, ctx_len_dev,
+                     out_dev, lse_dev, 0, stream);
+}
+
+extern "C" int pi_sparse_decode_attn_headwise(pi_ctx* ctx, int layer, int batch, const void* q_dev,
+                                              const void* pool_dev, const int32_t* sel_slots_dev,
+                                              const int32_t* sel_blocks_dev, const int32_t* sel_count_dev,
+                                              const int32_t* ctx_len_dev, void* out_dev, float* lse_dev,
+                                              void* stream) {
+    return attn_call(ctx, layer, batch, q_dev, pool_dev, sel_slots_dev, sel_blocks_dev, sel_count_dev, ctx_len_dev,
+                     out_dev, lse_dev, 1, stream);
 }
 
 static int append_call(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* k_new_dev, const void* v_new_dev,

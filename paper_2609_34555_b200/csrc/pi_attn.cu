@@ -37,8 +37,25 @@ struct AttnParams {
     unsigned int* counters;
     pi_status_ref st;
     int batch, Hq, Hkv, G, B, K, C, stages;
+    int headwise;                 // 1: sel_slots / sel_blocks are [batch][Hkv][K], sel_count [batch][Hkv]
     float scale_log2;
 };
+
+// Blocks of sequence s that the unit list walks: the selection's count, or, when every KV head has
+// its own selection, the largest count over the heads (a head with fewer blocks sees empty tiles).
+// Counts outside [0, K] read as 0 (the main kernel reports them).
+__device__ __forceinline__ int blocks_of_seq(const AttnParams& p, int s) {
+    if (!p.headwise) {
+        const int n = p.sel_count[s];
+        return (n < 0 || n > p.K) ? 0 : n;
+    }
+    int n = 0;
+    for (int h = 0; h < p.Hkv; ++h) {
+        const int c = p.sel_count[s * p.Hkv + h];
+        if (c >= 0 && c <= p.K) n = max(n, c);
+    }
+    return n;
+}
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -129,9 +146,7 @@ attn_merge_kernel(AttnParams p, int main_ctas) {
     // units before this sequence, of this sequence, and in total
     int before = 0, mine = 0, total = 0;
     for (int s = threadIdx.x; s < p.batch; s += blockDim.x) {
-        int n = p.sel_count[s];
-        if (n < 0 || n > p.K) n = 0;
-        n *= SUB;
+        int n = blocks_of_seq(p, s) * SUB;
         total += n;
         if (s < seq) before += n;
         if (s == seq) mine = n;
@@ -214,7 +229,12 @@ attn_merge_kernel(AttnParams p, int main_ctas) {
     }
 }
 
-template <int NT>
+// HW = false: one selection per sequence, a stage is one TMA box pair covering all KV heads of a block.
+// HW = true: every KV head has its own selection (the headwise strategy of Sec. 4.4.1): a stage holds,
+// for each head, the (K, V) fragment of that head's own j-th selected block, fetched with a box of two
+// rows of the head dimension (pool_map then has box {64, 16, 2, 1}); consumer warp h sees the same stage
+// layout either way.
+template <int NT, bool HW>
 __global__ void __launch_bounds__(288, 1)
 attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
     extern __shared__ unsigned char smem_dyn[];
@@ -223,8 +243,8 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
     const uint32_t ring = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     unsigned char* after_ring = smem_dyn + (ring - smem_u32(smem_dyn)) + static_cast<size_t>(p.stages) * stage_bytes;
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(after_ring);      // full[8], empty[8], seg
-    int* s_nvalid = reinterpret_cast<int*>(bars + 2 * ATTN_MAX_STAGES + 1);            // [8]
-    int* s_abort = s_nvalid + ATTN_MAX_STAGES;
+    int* s_nvalid = reinterpret_cast<int*>(bars + 2 * ATTN_MAX_STAGES + 1);            // [8 stages][8 heads]
+    int* s_abort = s_nvalid + ATTN_MAX_STAGES * 8;
     int* s_last = s_abort + 1;
     int2* s_meta = reinterpret_cast<int2*>(s_last + 1);                                // [ATTN_META_UNITS] {slot row, sub*16 | nvalid<<8}
     int* s_pref = reinterpret_cast<int*>(s_meta + ATTN_META_UNITS);                    // [batch + 1]
@@ -237,12 +257,14 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
 
     // ---- unit prefix over sequences (every CTA computes the same table)
     for (int s = tid; s < p.batch; s += blockDim.x) {
-        int n = p.sel_count[s];
-        if (n < 0 || n > p.K) {
-            if (blockIdx.x == 0) pi_report(p.st, PI_ERR_CAPACITY, PI_STAGE_ATTN, s, n, p.K);
-            n = 0;
+        if (blockIdx.x == 0) {
+            const int lists = HW ? p.Hkv : 1;
+            for (int i = 0; i < lists; ++i) {
+                const int n = p.sel_count[s * lists + i];
+                if (n < 0 || n > p.K) pi_report(p.st, PI_ERR_CAPACITY, PI_STAGE_ATTN, s, n, p.K);
+            }
         }
-        s_pref[s + 1] = n * SUB;
+        s_pref[s + 1] = blocks_of_seq(p, s) * SUB;
     }
     if (tid == 0) {
         s_pref[0] = 0;
@@ -290,19 +312,32 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
 
     // ---- metadata of this CTA's units: global row of the slot, token offset, valid tokens.
     // Staged up front by all threads so the producer never waits on a dependent global load.
-    auto unit_meta = [&](int u, int seq) -> int2 {
+    // hh: the KV head whose list is read (ignored when all heads share one selection)
+    auto unit_meta = [&](int u, int seq, int hh) -> int2 {
         const int r = u - s_pref[seq], j = r / SUB, sub = r - j * SUB;
-        int slot = p.sel_slots[static_cast<size_t>(seq) * p.K + j];
-        const int blk = p.sel_blocks[static_cast<size_t>(seq) * p.K + j];
-        if (slot < 0 || slot >= p.C) {
-            pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_ATTN, seq, j, slot);
-            slot = 0;
+        const size_t list = HW ? static_cast<size_t>(seq) * p.Hkv + hh : static_cast<size_t>(seq);
+        int jj = j;
+        bool empty = false;
+        if (HW) {                                    // a head with a shorter list: an empty tile of its first block
+            const int cnt = p.sel_count[list];
+            if (cnt < 0 || cnt > p.K || j >= cnt) { empty = true; jj = 0; }
         }
-        const int nvalid = blk < 0 ? 0 : max(0, min(16, p.ctx_len[seq] - (blk * p.B + sub * 16)));
+        int slot = p.sel_slots[list * p.K + jj];
+        const int blk = p.sel_blocks[list * p.K + jj];
+        if (slot < 0 || slot >= p.C) {
+            if (!empty) pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_ATTN, seq, j, slot);
+            slot = 0;
+            empty = HW ? true : empty;
+        }
+        const int nvalid = (blk < 0 || empty) ? 0 : max(0, min(16, p.ctx_len[seq] - (blk * p.B + sub * 16)));
         return make_int2(seq * p.C + slot, (sub * 16) | (nvalid << 8));
     };
-    for (int i = tid; i < u1 - u0 && i < ATTN_META_UNITS; i += blockDim.x)
-        s_meta[i] = unit_meta(u0 + i, seq_of_unit(s_pref, p.batch, u0 + i));
+    const int meta_per_unit = HW ? p.Hkv : 1;
+    const int meta_units = ATTN_META_UNITS / meta_per_unit;
+    for (int i = tid; i < (u1 - u0) * meta_per_unit && i < meta_units * meta_per_unit; i += blockDim.x) {
+        const int ui = i / meta_per_unit, hh = i - ui * meta_per_unit;
+        s_meta[i] = unit_meta(u0 + ui, seq_of_unit(s_pref, p.batch, u0 + ui), hh);
+    }
     __syncthreads();
 
     if (warp == p.Hkv) {
@@ -311,14 +346,29 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
             int seq = seq_of_unit(s_pref, p.batch, u0);
             for (int u = u0, it = 0; u < u1; ++u, ++it) {
                 while (u >= s_pref[seq + 1]) ++seq;
-                const int2 md = it < ATTN_META_UNITS ? s_meta[it] : unit_meta(u, seq);
                 const int st = it % p.stages, round = it / p.stages;
                 if (round > 0 && !mbar_wait(bar_empty + 8 * st, (round - 1) & 1, s_abort)) break;
-                s_nvalid[st] = md.y >> 8;
                 const uint32_t dst = ring + st * stage_bytes;
-                mbar_expect_tx(bar_full + 8 * st, stage_bytes);
-                tma_load_4d(dst, &pool_map, bar_full + 8 * st, 0, md.y & 0xff, 0, md.x);
-                tma_load_4d(dst + half_bytes, &pool_map, bar_full + 8 * st, 64, md.y & 0xff, 0, md.x);
+                // valid-token counts are written before the arrive below, which publishes them
+                if (HW) {
+                    int rows[8], offs[8];
+                    for (int hh = 0; hh < p.Hkv; ++hh) {
+                        const int2 md = it < meta_units ? s_meta[it * p.Hkv + hh] : unit_meta(u, seq, hh);
+                        s_nvalid[st * 8 + hh] = md.y >> 8;
+                        rows[hh] = md.x; offs[hh] = md.y & 0xff;
+                    }
+                    mbar_expect_tx(bar_full + 8 * st, stage_bytes);
+                    for (int hh = 0; hh < p.Hkv; ++hh) {
+                        tma_load_4d(dst + hh * 4096, &pool_map, bar_full + 8 * st, 0, offs[hh], 2 * hh, rows[hh]);
+                        tma_load_4d(dst + half_bytes + hh * 4096, &pool_map, bar_full + 8 * st, 64, offs[hh], 2 * hh, rows[hh]);
+                    }
+                } else {
+                    const int2 md = it < meta_units ? s_meta[it] : unit_meta(u, seq, 0);
+                    s_nvalid[st * 8] = md.y >> 8;
+                    mbar_expect_tx(bar_full + 8 * st, stage_bytes);
+                    tma_load_4d(dst, &pool_map, bar_full + 8 * st, 0, md.y & 0xff, 0, md.x);
+                    tma_load_4d(dst + half_bytes, &pool_map, bar_full + 8 * st, 64, md.y & 0xff, 0, md.x);
+                }
             }
         }
         return;
@@ -359,7 +409,7 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
       for (; u < seg_end; ++u, ++it) {
         const int st = it % p.stages;
         if (!mbar_wait(bar_full + 8 * st, (it / p.stages) & 1, s_abort)) { alive = false; break; }
-        const int nvalid = s_nvalid[st];
+        const int nvalid = s_nvalid[st * 8 + (HW ? h : 0)];
         const uint32_t base = ring + st * stage_bytes;
 
         // ---- S^T = K q^T
@@ -485,18 +535,19 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
 
 int pi_launch_attn(pi_ctx* c, int batch, const void* q, const void* pool, const int32_t* sel_slots,
                    const int32_t* sel_blocks, const int32_t* sel_count, const int32_t* ctx_len, void* out,
-                   float* lse, cudaStream_t stream) {
+                   float* lse, int headwise, cudaStream_t stream) {
     const pi_config& cfg = c->cfg;
     if (cfg.n_kv_heads > 8) return PI_ERR_UNSUPPORTED_DIM;
     const long long n_slots = static_cast<long long>(batch) * cfg.pool_slots;
-    if (c->pool_map_ptr != pool || c->pool_map_slots != n_slots) {
+    // the map is rebuilt when the pool, its size or the box (all heads / one head per load) changes
+    if (c->pool_map_ptr != pool || c->pool_map_slots != n_slots || c->pool_map_headwise != headwise) {
         typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                       const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                       CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
         const cuuint64_t B = cfg.block_tokens, hk = 2ull * cfg.n_kv_heads;
         cuuint64_t gdim[4] = {PI_HEAD_DIM, B, hk, static_cast<cuuint64_t>(n_slots)};
         cuuint64_t gstride[3] = {PI_HEAD_DIM * 2ull, B * PI_HEAD_DIM * 2ull, hk * B * PI_HEAD_DIM * 2ull};
-        cuuint32_t box[4] = {64, 16, static_cast<cuuint32_t>(hk), 1};
+        cuuint32_t box[4] = {64, 16, headwise ? 2u : static_cast<cuuint32_t>(hk), 1};
         cuuint32_t estr[4] = {1, 1, 1, 1};
         CUresult r = reinterpret_cast<encode_fn>(c->encode_tiled_fn)(
             &c->pool_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), gdim, gstride, box, estr,
@@ -505,6 +556,7 @@ int pi_launch_attn(pi_ctx* c, int batch, const void* q, const void* pool, const 
         if (r != CUDA_SUCCESS) { c->pool_map_ptr = nullptr; return PI_ERR_CUDA; }
         c->pool_map_ptr = pool;
         c->pool_map_slots = n_slots;
+        c->pool_map_headwise = headwise;
     }
     AttnParams p;
     p.q = static_cast<const __nv_bfloat16*>(q);
@@ -515,21 +567,24 @@ int pi_launch_attn(pi_ctx* c, int batch, const void* q, const void* pool, const 
     p.st = pi_status_of(c);
     p.batch = batch; p.Hq = cfg.n_q_heads; p.Hkv = cfg.n_kv_heads; p.G = cfg.n_q_heads / cfg.n_kv_heads;
     p.B = cfg.block_tokens; p.K = cfg.budget_blocks; p.C = cfg.pool_slots;
+    p.headwise = headwise ? 1 : 0;
     const int stage_bytes = cfg.n_kv_heads * 8192;
     int stages = ATTN_SMEM_BUDGET / stage_bytes;
     if (stages > ATTN_MAX_STAGES) stages = ATTN_MAX_STAGES;
     p.stages = stages;
     p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(PI_HEAD_DIM));
     const size_t smem = 1024 + static_cast<size_t>(stages) * stage_bytes + (2 * ATTN_MAX_STAGES + 1) * 8 +
-                        (ATTN_MAX_STAGES + 2) * 4 + ATTN_META_UNITS * 8 + (static_cast<size_t>(batch) + 1) * 4 + 16;
+                        (ATTN_MAX_STAGES * 8 + 2) * 4 + ATTN_META_UNITS * 8 + (static_cast<size_t>(batch) + 1) * 4 + 16;
     const int threads = (cfg.n_kv_heads + 1) * 32;
-    if (p.G <= 8) {
-        PI_CUDA_TRY(cudaFuncSetAttribute(attn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-        attn_kernel<1><<<c->attn_ctas, threads, smem, stream>>>(c->pool_map, p);
-    } else {
-        PI_CUDA_TRY(cudaFuncSetAttribute(attn_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-        attn_kernel<2><<<c->attn_ctas, threads, smem, stream>>>(c->pool_map, p);
-    }
+    auto launch = [&](auto kernel) -> int {
+        PI_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+        kernel<<<c->attn_ctas, threads, smem, stream>>>(c->pool_map, p);
+        return PI_OK;
+    };
+    int rc;
+    if (headwise) rc = p.G <= 8 ? launch(attn_kernel<1, true>) : launch(attn_kernel<2, true>);
+    else rc = p.G <= 8 ? launch(attn_kernel<1, false>) : launch(attn_kernel<2, false>);
+    if (rc != PI_OK) return rc;
     PI_CUDA_TRY(cudaGetLastError());
     // merge of the split sequences: may start early, synchronises on the grid above by itself
     cudaLaunchConfig_t lc = {};

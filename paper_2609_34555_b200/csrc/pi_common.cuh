@@ -38,6 +38,7 @@ struct pi_ctx {
     CUtensorMap pool_map;
     const void* pool_map_ptr;
     long long pool_map_slots;
+    int pool_map_headwise;       // box of the cached map: all KV heads of a block (0) or one head (1)
     void* encode_tiled_fn;
 };
 
@@ -88,7 +89,7 @@ int pi_launch_recall(pi_ctx*, int n_lists, int lists_per_seq, const void* host_k
                      const int32_t* page_table, int64_t page_stride, int32_t n_pages, cudaStream_t);
 int pi_launch_attn(pi_ctx*, int batch, const void* q, const void* pool, const int32_t* sel_slots,
                    const int32_t* sel_blocks, const int32_t* sel_count, const int32_t* ctx_len,
-                   void* out, float* lse, cudaStream_t);
+                   void* out, float* lse, int headwise, cudaStream_t);
 int pi_launch_append(pi_ctx*, int h_star, int batch, uint32_t step, const void* k_new, const void* v_new,
                      const int32_t* ctx_len, void* host_kv, int64_t host_stride, void* pool, int32_t* table,
                      int32_t* slot_block, uint32_t* slot_stamp, void* digest, const int32_t* page_table,

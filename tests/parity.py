@@ -381,7 +381,8 @@ def run_append_and_compare(cfg, steps: int, ctx_len0, layer: int = 0) -> dict:
 
 def run_strategies_and_compare(cfg, steps: int = 2, layer: int = 0) -> dict:
     """The averaged and the headwise selection strategies: scores and selections against the
-    oracle, then (headwise) per-head diff and per-head fragment recall, pool bytes bit-exact."""
+    oracle, then (headwise) per-head diff and per-head fragment recall, pool bytes bit-exact, and
+    attention of every KV head's query group over that head's own selection."""
     from paper_2609_34555_b200 import PulseInfer
 
     dev = torch.device("cuda:0")
@@ -428,6 +429,10 @@ def run_strategies_and_compare(cfg, steps: int = 2, layer: int = 0) -> dict:
     lst = torch.zeros((R, K, 4), dtype=torch.int32, device=dev)
     lcnt = torch.zeros((R,), dtype=torch.int32, device=dev)
     pool = torch.zeros((cfg.batch, C, Hkv, 2, cfg.block_tokens, cfg.head_dim), dtype=torch.bfloat16, device=dev)
+    out = torch.zeros((cfg.batch, cfg.n_q_heads, cfg.head_dim), dtype=torch.bfloat16, device=dev)
+    lse = torch.zeros((cfg.batch, cfg.n_q_heads), dtype=torch.float32, device=dev)
+    G = cfg.group
+    stats["attn_max_abs"] = 0.0
     ctx_rows = ctx_d.repeat_interleave(Hkv).contiguous()
     res_rows = np.repeat(case.resident, Hkv, axis=0)                       # every head starts with the same hot set
     pi.table_init(torch.from_numpy(res_rows).to(dev), table, slot_block, slot_stamp)
@@ -440,6 +445,16 @@ def run_strategies_and_compare(cfg, steps: int = 2, layer: int = 0) -> dict:
         ok = res_rows[r] >= 0
         o_table[r, res_rows[r][ok]] = np.nonzero(ok)[0]
     frag, blockb = cfg.frag_bytes, cfg.block_bytes
+    # the initial hot set really sits in the pool (same blocks for every head), on both sides
+    fill = torch.zeros((cfg.batch, C, 4), dtype=torch.int32)
+    fcnt = torch.zeros((cfg.batch,), dtype=torch.int32)
+    for s in range(cfg.batch):
+        ok = np.nonzero(case.resident[s] >= 0)[0]
+        for i, slot in enumerate(ok):
+            fill[s, i] = torch.tensor([int(case.resident[s][slot]), int(slot), 1, i], dtype=torch.int32)
+            o_pool[s, slot] = kvb[s, case.resident[s][slot]]
+        fcnt[s] = len(ok)
+    pi.recall_gather_scatter(layer, case.kv, pool, fill.to(dev), fcnt.to(dev))
     for t in range(steps):
         step = t + 1
         q_d, qb = case.q[t].to(dev), oracle.bits(case.q[t])
@@ -447,8 +462,10 @@ def run_strategies_and_compare(cfg, steps: int = 2, layer: int = 0) -> dict:
         pi.diff_misses(layer, step, ctx_rows, hsel, hcnt, table, slot_block, slot_stamp, slots, lst, lcnt)
         pi.recall_gather_scatter(layer, case.kv, pool, lst, lcnt, lists_per_seq=Hkv, unit_bytes=frag,
                                  unit_stride=blockb, list_offset=frag)
+        pi.sparse_decode_attn(layer, q_d, pool, slots, hsel, hcnt, ctx_d, out, lse, headwise=True)
         torch.cuda.synchronize()
         assert pi.status()[0] == 0, pi.status()
+        g_out, g_lse = out.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
         g_sc, g_sel, g_cnt = hsc.cpu().numpy(), hsel.cpu().numpy(), hcnt.cpu().numpy()
         g_slots, g_lst, g_lcnt = slots.cpu().numpy(), lst.cpu().numpy(), lcnt.cpu().numpy()
         for s in range(cfg.batch):
@@ -469,6 +486,21 @@ def run_strategies_and_compare(cfg, steps: int = 2, layer: int = 0) -> dict:
                 stats["misses"] += len(pairs)
         assert np.array_equal(table.cpu().numpy(), o_table)
         assert np.array_equal(oracle.bits(pool.cpu()), o_pool), "per-head fragments in the pool"
+        # attention: the query heads of KV head h over head h's own blocks, read from the oracle's pool
+        # through the oracle's slots and, independently, from the host copy through the block indices
+        for s in range(cfg.batch):
+            for h in range(Hkv):
+                r = s * Hkv + h
+                ref, ref_lse = oracle.attention(qb[s], o_pool[s], g_slots[r], g_sel[r], int(g_cnt[r]), int(case.ctx_len[s]),
+                                                cfg.block_tokens, Hkv)
+                via_host, _ = oracle.attention(qb[s], kvb[s], g_sel[r], g_sel[r], int(g_cnt[r]), int(case.ctx_len[s]),
+                                               cfg.block_tokens, Hkv)
+                rows = slice(h * G, (h + 1) * G)
+                assert np.array_equal(ref[rows], via_host[rows]), "byte invariant seen through attention"
+                err = np.abs(g_out[s, rows] - ref[rows])
+                stats["attn_max_abs"] = max(stats["attn_max_abs"], float(err.max()))
+                assert np.all(err <= np.maximum(ATTN_MAX_ABS, np.abs(ref[rows]) * 2.0 ** -8)) and err.mean() <= ATTN_MEAN_ABS
+                np.testing.assert_allclose(g_lse[s, rows], ref_lse[rows], rtol=1e-3, atol=1e-3)
     # heads really choose differently (the fragmentation the shared selection avoids)
     stats["distinct_head_selections"] = len({tuple(g_sel[h].tolist()) for h in range(Hkv)})
     pi.close()

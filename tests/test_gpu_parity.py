@@ -427,3 +427,57 @@ def test_double_buffered_host_stepping_matches_plain_stepping():
         pi.close()
     for t in range(steps):
         assert torch.equal(outs[0][t].view(torch.int16), outs[1][t].view(torch.int16)), f"step {t}"
+
+
+def test_headwise_attention_with_unequal_and_empty_head_lists():
+    """Every KV head attends over its own list; lists of one sequence differ in length, one is empty,
+    the last block is partial.  Pool slot i holds block i, so slots and blocks coincide."""
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2609_34555_b200 import PulseInfer
+    from tests.parity import ATTN_MAX_ABS, ATTN_MEAN_ABS
+    from workloads import generate as gen
+    cfg = tiny_config(batch=3, ctx=16 * 37 + 5, n_q_heads=16, n_kv_heads=4, budget_blocks=20, resident_frac=1.0)
+    nb, Hkv, K, G = cfg.n_blocks, cfg.n_kv_heads, cfg.budget_blocks, cfg.group
+    assert cfg.pool_slots >= nb
+    pi = PulseInfer.from_workload(cfg)
+    kv = gen.make_kv(cfg, 0)
+    kvb = oracle.bits(kv)
+    pool = torch.zeros((cfg.batch, cfg.pool_slots) + tuple(kv.shape[2:]), dtype=torch.bfloat16)
+    pool[:, :nb] = kv
+    q = gen.make_queries(cfg, 0, 1)[0]
+    qb = oracle.bits(q)
+    rng = np.random.default_rng(5)
+    sel = np.full((cfg.batch, Hkv, K), -1, np.int32)
+    cnt = np.zeros((cfg.batch, Hkv), np.int32)
+    for s in range(cfg.batch):
+        for h in range(Hkv):
+            n = [K, 7, 0, 13][(s + h) % 4]
+            rows = np.sort(rng.choice(nb, size=n, replace=False)).astype(np.int32)
+            if n and (s + h) % 2 == 0:
+                rows[-1] = nb - 1                                   # the partial last block
+                rows = np.unique(rows)
+            sel[s, h, : len(rows)] = rows
+            cnt[s, h] = len(rows)
+    ctx = np.full(cfg.batch, cfg.ctx, np.int32)
+    out = torch.zeros((cfg.batch, cfg.n_q_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros((cfg.batch, cfg.n_q_heads), dtype=torch.float32, device="cuda")
+    sel_d = torch.from_numpy(sel).cuda()
+    pi.sparse_decode_attn(0, q.cuda(), pool.cuda(), sel_d, sel_d, torch.from_numpy(cnt).cuda(),
+                          torch.from_numpy(ctx).cuda(), out, lse, headwise=True)
+    torch.cuda.synchronize()
+    assert pi.status()[0] == 0, pi.status()
+    g_out, g_lse = out.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
+    for s in range(cfg.batch):
+        for h in range(Hkv):
+            rows = slice(h * G, (h + 1) * G)
+            if cnt[s, h] == 0:
+                assert np.all(g_out[s, rows] == 0) and np.all(np.isneginf(g_lse[s, rows]))
+                continue
+            ref, ref_lse = oracle.attention(qb[s], kvb[s], sel[s, h], sel[s, h], int(cnt[s, h]), cfg.ctx,
+                                            cfg.block_tokens, Hkv)
+            err = np.abs(g_out[s, rows] - ref[rows])
+            assert np.all(err <= np.maximum(ATTN_MAX_ABS, np.abs(ref[rows]) * 2.0 ** -8)) and err.mean() <= ATTN_MEAN_ABS
+            np.testing.assert_allclose(g_lse[s, rows], ref_lse[rows], rtol=1e-3, atol=1e-3)
+    pi.close()
