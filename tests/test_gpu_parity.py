@@ -481,3 +481,49 @@ def test_headwise_attention_with_unequal_and_empty_head_lists():
             assert np.all(err <= np.maximum(ATTN_MAX_ABS, np.abs(ref[rows]) * 2.0 ** -8)) and err.mean() <= ATTN_MEAN_ABS
             np.testing.assert_allclose(g_lse[s, rows], ref_lse[rows], rtol=1e-3, atol=1e-3)
     pi.close()
+
+
+def test_layer_step_can_be_captured_into_a_cuda_graph_and_replayed():
+    """No call of the path synchronises the host or allocates: one layer-step (score/select, diff,
+    recall, attention) captured into a CUDA graph and replayed from the same starting state gives
+    the bits of the eager run."""
+    import torch
+    from paper_2609_34555_b200 import PulseInfer
+    from paper_2609_34555_b200.runner import LayerBuffers, RecallPath
+    from tests.parity import make_case
+    cfg = tiny_config(batch=4, ctx=2048, n_q_heads=16, n_kv_heads=4, budget_blocks=24, resident_frac=0.3)
+    case = make_case(cfg, steps=1)
+    dev = torch.device("cuda:0")
+    pi = PulseInfer.from_workload(cfg)
+    path = RecallPath(pi)
+    buf = LayerBuffers(pi, cfg.batch, dev)
+    ctx_d = torch.from_numpy(case.ctx_len).to(dev)
+    path.prepare_layer(0, buf, case.kv, ctx_d, torch.from_numpy(case.resident).to(dev))
+    q_d = case.q[0].to(dev)
+    out = torch.zeros((cfg.batch, cfg.n_q_heads, cfg.head_dim), dtype=torch.bfloat16, device=dev)
+    lse = torch.zeros((cfg.batch, cfg.n_q_heads), dtype=torch.float32, device=dev)
+    torch.cuda.synchronize()
+    state = [t.clone() for t in (buf.block_table, buf.slot_block, buf.slot_stamp, buf.pool)]
+
+    path.layer_step(0, 1, buf, q_d, ctx_d, case.kv, out, lse)          # eager (also warms every launch path up)
+    torch.cuda.synchronize()
+    want = [t.clone() for t in (out, lse, buf.sel_blocks, buf.sel_slots, buf.recall_count, buf.block_table,
+                                buf.slot_stamp, buf.pool)]
+    assert int(buf.recall_count.sum()) > 0
+
+    for t, s in zip((buf.block_table, buf.slot_block, buf.slot_stamp, buf.pool), state):
+        t.copy_(s)
+    out.zero_(); lse.zero_()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        path.layer_step(0, 1, buf, q_d, ctx_d, case.kv, out, lse)
+    torch.cuda.synchronize()
+    assert float(out.float().abs().sum()) == 0.0                       # capture records, it does not run
+    graph.replay()
+    torch.cuda.synchronize()
+    assert pi.status()[0] == 0, pi.status()
+    got = (out, lse, buf.sel_blocks, buf.sel_slots, buf.recall_count, buf.block_table, buf.slot_stamp, buf.pool)
+    for g, w in zip(got, want):
+        assert torch.equal(g.view(torch.int16) if g.dtype == torch.bfloat16 else g, w.view(torch.int16) if w.dtype == torch.bfloat16 else w)
+    pi.close()
