@@ -156,6 +156,15 @@ int pi_diff_misses(pi_ctx* ctx, int layer, int batch, uint32_t step, const int32
                    int32_t* sel_slots_dev, pi_extent* recall_list_dev, int32_t* recall_count_dev,
                    void* stream);
 
+/* The same with the step number read from device memory when the kernel runs (one uint32, > 0), so
+ * that a CUDA graph holding the call can be replayed for later steps: the caller advances *step_dev
+ * between replays (in the graph or outside).  The paper has no counterpart. */
+int pi_diff_misses_devstep(pi_ctx* ctx, int layer, int batch, const uint32_t* step_dev,
+                           const int32_t* ctx_len_dev, const int32_t* sel_blocks_dev,
+                           const int32_t* sel_count_dev, int32_t* block_table_dev, int32_t* slot_block_dev,
+                           uint32_t* slot_stamp_dev, int32_t* sel_slots_dev, pi_extent* recall_list_dev,
+                           int32_t* recall_count_dev, void* stream);
+
 /* Step 3 of the workflow (Sec. 2.2; Sec. 4.4.2 gather-scatter transfer): copy every
  * extent of every list from the pinned host store into the HBM pool, byte for byte.
  * The GPU pulls the data itself with wide loads; counts and lists are read from

@@ -141,20 +141,38 @@ extern "C" int pi_score_select_strategy(pi_ctx* ctx, int strategy, int layer, in
                                            static_cast<cudaStream_t>(stream));
 }
 
+static int diff_call(pi_ctx* ctx, int layer, int batch, uint32_t step, const uint32_t* step_dev,
+                     const int32_t* ctx_len_dev, const int32_t* sel_blocks_dev, const int32_t* sel_count_dev,
+                     int32_t* block_table_dev, int32_t* slot_block_dev, uint32_t* slot_stamp_dev,
+                     int32_t* sel_slots_dev, pi_extent* recall_list_dev, int32_t* recall_count_dev, void* stream) {
+    int rc = check_call(ctx, layer, batch);
+    if (rc != PI_OK) return rc;
+    if (!ctx_len_dev || !sel_blocks_dev || !sel_count_dev || !block_table_dev || !slot_block_dev ||
+        !slot_stamp_dev || !sel_slots_dev || !recall_list_dev || !recall_count_dev || (!step_dev && step == 0))
+        return PI_ERR_INVALID_ARG;
+    if (!pi_aligned16(recall_list_dev)) return PI_ERR_BAD_ALIGN;
+    return pi_launch_diff(ctx, batch, step, step_dev, ctx_len_dev, sel_blocks_dev, sel_count_dev, block_table_dev,
+                          slot_block_dev, slot_stamp_dev, sel_slots_dev, recall_list_dev, recall_count_dev,
+                          static_cast<cudaStream_t>(stream));
+}
+
 extern "C" int pi_diff_misses(pi_ctx* ctx, int layer, int batch, uint32_t step, const int32_t* ctx_len_dev,
                               const int32_t* sel_blocks_dev, const int32_t* sel_count_dev,
                               int32_t* block_table_dev, int32_t* slot_block_dev, uint32_t* slot_stamp_dev,
                               int32_t* sel_slots_dev, pi_extent* recall_list_dev, int32_t* recall_count_dev,
                               void* stream) {
-    int rc = check_call(ctx, layer, batch);
-    if (rc != PI_OK) return rc;
-    if (!ctx_len_dev || !sel_blocks_dev || !sel_count_dev || !block_table_dev || !slot_block_dev ||
-        !slot_stamp_dev || !sel_slots_dev || !recall_list_dev || !recall_count_dev || step == 0)
-        return PI_ERR_INVALID_ARG;
-    if (!pi_aligned16(recall_list_dev)) return PI_ERR_BAD_ALIGN;
-    return pi_launch_diff(ctx, batch, step, ctx_len_dev, sel_blocks_dev, sel_count_dev, block_table_dev,
-                          slot_block_dev, slot_stamp_dev, sel_slots_dev, recall_list_dev, recall_count_dev,
-                          static_cast<cudaStream_t>(stream));
+    return diff_call(ctx, layer, batch, step, nullptr, ctx_len_dev, sel_blocks_dev, sel_count_dev, block_table_dev,
+                     slot_block_dev, slot_stamp_dev, sel_slots_dev, recall_list_dev, recall_count_dev, stream);
+}
+
+extern "C" int pi_diff_misses_devstep(pi_ctx* ctx, int layer, int batch, const uint32_t* step_dev,
+                                      const int32_t* ctx_len_dev, const int32_t* sel_blocks_dev,
+                                      const int32_t* sel_count_dev, int32_t* block_table_dev,
+                                      int32_t* slot_block_dev, uint32_t* slot_stamp_dev, int32_t* sel_slots_dev,
+                                      pi_extent* recall_list_dev, int32_t* recall_count_dev, void* stream) {
+    if (!step_dev) return PI_ERR_INVALID_ARG;
+    return diff_call(ctx, layer, batch, 0, step_dev, ctx_len_dev, sel_blocks_dev, sel_count_dev, block_table_dev,
+                     slot_block_dev, slot_stamp_dev, sel_slots_dev, recall_list_dev, recall_count_dev, stream);
 }
 
 // Shared by the block-major and the paged entry point (page_table == nullptr: block-major).

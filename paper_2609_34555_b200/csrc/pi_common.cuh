@@ -80,7 +80,7 @@ int pi_launch_score_select(pi_ctx*, int h_star, int batch, const void* q, const 
 int pi_launch_score_select_strategy(pi_ctx*, int strategy, int batch, const void* q, const void* digest_all,
                                     const int32_t* ctx_len, int32_t* sel, int32_t* sel_count, float* scores,
                                     unsigned int* counters, cudaStream_t);
-int pi_launch_diff(pi_ctx*, int batch, uint32_t step, const int32_t* ctx_len, const int32_t* sel,
+int pi_launch_diff(pi_ctx*, int batch, uint32_t step, const uint32_t* step_dev, const int32_t* ctx_len, const int32_t* sel,
                    const int32_t* sel_count, int32_t* table, int32_t* slot_block, uint32_t* slot_stamp,
                    int32_t* sel_slots, pi_extent* list, int32_t* count, cudaStream_t);
 int pi_launch_recall(pi_ctx*, int n_lists, int lists_per_seq, const void* host_kv, int64_t host_stride,

@@ -31,6 +31,7 @@ struct DiffParams {
     pi_status_ref st;
     unsigned long long* stats;
     uint32_t step;
+    const uint32_t* step_dev;      // when set, the step is read from device memory (a captured graph replays with a new step)
     int B, K, C, Cpad, n_sink, n_local, max_blocks;
 };
 
@@ -57,6 +58,7 @@ __device__ __forceinline__ int ordered_pos(bool flag, int& base, int* warp_tot) 
 __global__ void __launch_bounds__(DIFF_THREADS)
 diff_kernel(DiffParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    const uint32_t step = p.step_dev ? *p.step_dev : p.step;
     unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);       // [Cpad]
     int32_t* s_sel = reinterpret_cast<int32_t*>(keys + p.Cpad);                         // [K]
     int32_t* s_slot = s_sel + p.K;                                                      // [K] slot of sel[j]
@@ -199,7 +201,7 @@ diff_kernel(DiffParams p) {
         int slot = -1;
         if (j < cnt) {
             slot = s_slot[j];
-            if (slot >= 0 && !too_small) slot_stamp[slot] = p.step;
+            if (slot >= 0 && !too_small) slot_stamp[slot] = step;
         }
         sel_slots[j] = slot;
     }
@@ -246,7 +248,7 @@ diff_kernel(DiffParams p) {
 
 }  // namespace
 
-int pi_launch_diff(pi_ctx* c, int batch, uint32_t step, const int32_t* ctx_len, const int32_t* sel,
+int pi_launch_diff(pi_ctx* c, int batch, uint32_t step, const uint32_t* step_dev, const int32_t* ctx_len, const int32_t* sel,
                    const int32_t* sel_count, int32_t* table, int32_t* slot_block, uint32_t* slot_stamp,
                    int32_t* sel_slots, pi_extent* list, int32_t* count, cudaStream_t stream) {
     DiffParams p;
@@ -256,6 +258,7 @@ int pi_launch_diff(pi_ctx* c, int batch, uint32_t step, const int32_t* ctx_len, 
     p.st = pi_status_of(c);
     p.stats = c->stats_dev;
     p.step = step;
+    p.step_dev = step_dev;
     p.B = c->cfg.block_tokens; p.K = c->cfg.budget_blocks; p.C = c->cfg.pool_slots;
     int cpad = 2;
     while (cpad < p.C) cpad <<= 1;

@@ -224,6 +224,7 @@ class DecodeSession:
         self.out = torch.zeros((n_layers, batch, c.n_q_heads, c.head_dim), dtype=torch.bfloat16, device=device)
         self.ctx_len = torch.zeros((batch,), dtype=torch.int32, device=device)
         self.ctx_prev = torch.zeros((batch,), dtype=torch.int32, device=device)     # length before the step's append
+        self.step_dev = torch.zeros((1,), dtype=torch.int32, device=device)         # step number of graph replays
         self.main = torch.cuda.current_stream(self.device)
         self.side = torch.cuda.Stream(self.device)
         self.side2 = torch.cuda.Stream(self.device)
@@ -270,7 +271,7 @@ class DecodeSession:
 
     def decode_step(self, q: torch.Tensor, overlapped: bool = True, timer: Optional[StageTimer] = None,
                     resident_script: Optional[torch.Tensor] = None, new_kv=None,
-                    out: Optional[torch.Tensor] = None) -> torch.Tensor:
+                    out: Optional[torch.Tensor] = None, capturing: bool = False) -> torch.Tensor:
         """q: device bf16 [n_layers][batch][Hq][D].  Returns `out` (default self.out, [n_layers][batch][Hq][D]);
         valid once the current stream has caught up.  resident_script (int32 [n_layers][batch][C]):
         workloads with scripted miss counts reset each layer's tables to these hot-set contents
@@ -290,6 +291,11 @@ class DecodeSession:
         if overlapped:
             self._ev_start.record(main)
             sel_s.wait_event(self._ev_start)
+        if capturing:
+            # inside a graph the step number lives on the device and advances with every replay
+            with torch.cuda.stream(sel_s):
+                self.step_dev += 1
+            step = self.step_dev
         if new_kv is not None:
             with torch.cuda.stream(sel_s):
                 self.ctx_prev.copy_(self.ctx_len)
@@ -305,10 +311,14 @@ class DecodeSession:
                 tm = None
             else:
                 ev_attn_new = None
-            if overlapped and step > 1:
+            if overlapped and not capturing and self.step_count > 1:
                 sel_s.wait_event(self._ev_attn[l])         # last step's attention still reads this layer's lists and pool
             if ev_attn_new is not None:
                 self._ev_attn[l] = ev_attn_new
+            if capturing:                                  # events of a capture live in the graph only
+                evd, evr, eva = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
+            else:
+                evd, evr, eva = self._ev_diff[l], self._ev_recall[l], self._ev_attn[l]
             if resident_script is not None:
                 pi.table_init(resident_script[l], b.block_table, b.slot_block, b.slot_stamp, stream=sel_s)
             if new_kv is not None:
@@ -324,26 +334,48 @@ class DecodeSession:
                            b.slot_stamp, b.sel_slots, b.recall_list, b.recall_count, stream=sel_s)
             t2 = tm.mark(sel_s) if tm and tm.wants("diff") else None
             if overlapped:
-                self._ev_diff[l].record(sel_s)
-                rec_s.wait_event(self._ev_diff[l])
+                evd.record(sel_s)
+                rec_s.wait_event(evd)
             t2r = tm.mark(rec_s) if tm and tm.wants("recall") else None
             pi.recall_gather_scatter(l, host, b.pool, b.recall_list, b.recall_count, page_table=pt, stream=rec_s)
             t3 = tm.mark(rec_s) if tm and tm.wants("recall") else None
             if overlapped:
-                self._ev_recall[l].record(rec_s)
-                main.wait_event(self._ev_recall[l])
+                evr.record(rec_s)
+                main.wait_event(evr)
             t4 = tm.mark(main) if tm and tm.wants("attn") else None
             pi.sparse_decode_attn(l, q[l], b.pool, b.sel_slots, b.sel_blocks, b.sel_count, self.ctx_len,
                                   out[l], None, stream=main)
             t5 = tm.mark(main) if tm and tm.wants("attn") else None
             if overlapped:
-                self._ev_attn[l].record(main)
+                eva.record(main)
             if tm:
                 if t0 is not None: tm.add("score_select", t0, t1)
                 if t2 is not None: tm.add("diff", t1, t2)
                 if t2r is not None: tm.add("recall", t2r, t3)
                 if t4 is not None: tm.add("attn", t4, t5)
         return out
+
+    def capture_step(self, q_static: torch.Tensor, out: Optional[torch.Tensor] = None) -> "torch.cuda.CUDAGraph":
+        """Captures one pipelined decode step (all layers, all streams) into a CUDA graph that reads
+        its queries from `q_static` and its step number from device memory.  Replays continue the
+        session: call `graph.replay()` once per decode step after refreshing `q_static` (stream
+        order serialises consecutive replays, as consecutive decode steps are anyway).  Eager steps
+        and replays may be mixed; steps that append tokens or reset the tables stay eager."""
+        torch.cuda.synchronize(self.device)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.decode_step(q_static, overlapped=True, out=out, capturing=True)
+        self.step_count -= 1                              # the capture itself ran nothing
+        self._step_dev_shadow = None
+        return graph
+
+    def replay_step(self, graph: "torch.cuda.CUDAGraph") -> None:
+        """One decode step by replaying a graph from capture_step on the current stream."""
+        if getattr(self, "_step_dev_shadow", None) != self.step_count:
+            self.step_dev.fill_(self.step_count)          # eager steps ran in between: resynchronise the device counter
+        self.step_count += 1
+        self._step_dev_shadow = self.step_count           # the replay adds one on the device
+        graph.replay()
 
     def decode_steps_from_host(self, q_hosts, out_hosts, resident_scripts=None) -> None:
         """End-to-end form over several steps with the copies off the critical path: step i's queries

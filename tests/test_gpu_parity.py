@@ -527,3 +527,51 @@ def test_layer_step_can_be_captured_into_a_cuda_graph_and_replayed():
     for g, w in zip(got, want):
         assert torch.equal(g.view(torch.int16) if g.dtype == torch.bfloat16 else g, w.view(torch.int16) if w.dtype == torch.bfloat16 else w)
     pi.close()
+
+
+def test_graph_replayed_decode_steps_match_eager_steps():
+    """A whole pipelined decode step (three layers, all streams) captured once and replayed, with an
+    eager step mixed in: outputs, tables and stamps equal those of a session stepped eagerly."""
+    import torch
+    from paper_2609_34555_b200 import PulseInfer
+    from paper_2609_34555_b200.runner import DecodeSession
+    from workloads import generate as gen
+    cfg = tiny_config(batch=3, ctx=2048, n_q_heads=16, n_kv_heads=4, budget_blocks=24, resident_frac=0.3, n_layers=3)
+    steps = 6
+    results = []
+    for form in ("eager", "graph"):
+        pi = PulseInfer.from_workload(cfg)
+        sess = DecodeSession(pi, cfg.batch, cfg.n_layers)
+        sess.ctx_len.fill_(cfg.ctx)
+        for l in range(cfg.n_layers):
+            kv = gen.make_kv(cfg, l, device=sess.device)
+            sess.load_layer(l, kv, torch.from_numpy(gen.initial_resident(cfg, l)).to(sess.device))
+        q_all = torch.stack([gen.make_queries(cfg, l, steps, device=sess.device) for l in range(cfg.n_layers)], 1).contiguous()
+        got = []
+        if form == "eager":
+            for t in range(steps):
+                sess.decode_step(q_all[t])
+                torch.cuda.synchronize()
+                got.append(sess.out.cpu().clone())
+        else:
+            sess.decode_step(q_all[0])                     # step 1 eager (warms the launch paths up)
+            torch.cuda.synchronize()
+            got.append(sess.out.cpu().clone())
+            q_static = q_all[0].clone()
+            graph = sess.capture_step(q_static)
+            for t in range(1, steps):
+                if t == 3:                                 # an eager step between replays
+                    sess.decode_step(q_all[t])
+                else:
+                    q_static.copy_(q_all[t])
+                    sess.replay_step(graph)
+                torch.cuda.synchronize()
+                got.append(sess.out.cpu().clone())
+        assert pi.status()[0] == 0, pi.status()
+        state = [torch.stack([getattr(b, name).cpu() for b in sess.bufs]) for name in ("block_table", "slot_stamp", "sel_slots")]
+        results.append((got, state))
+        pi.close()
+    for t in range(steps):
+        assert torch.equal(results[0][0][t].view(torch.int16), results[1][0][t].view(torch.int16)), f"outputs of step {t}"
+    for a, b in zip(results[0][1], results[1][1]):
+        assert torch.equal(a, b)
