@@ -377,17 +377,29 @@ class DecodeSession:
         self._step_dev_shadow = self.step_count           # the replay adds one on the device
         graph.replay()
 
-    def decode_steps_from_host(self, q_hosts, out_hosts, resident_scripts=None) -> None:
+    def prepare_host_graph(self) -> None:
+        """Captures the graph decode_steps_from_host(use_graph=True) replays (synchronises; once)."""
+        if getattr(self, "_host_graph", None) is None:
+            self._q_static = torch.empty(self.out.shape, dtype=torch.bfloat16, device=self.device)
+            self._host_graph = self.capture_step(self._q_static)
+
+    def decode_steps_from_host(self, q_hosts, out_hosts, resident_scripts=None, use_graph: bool = False) -> None:
         """End-to-end form over several steps with the copies off the critical path: step i's queries
         (pinned host, [n_layers][batch][Hq][D]) are uploaded on a copy stream while step i-1 computes,
         step i's outputs are downloaded to out_hosts[i % len(out_hosts)] (pinned host) while step i+1
-        computes.  Queries and outputs are double-buffered on the device.  Returns once everything is
+        computes.  Queries and outputs are double-buffered on the device.  With use_graph the step
+        itself is a replay of the graph from capture_step (device-to-device copies move the queries
+        into, and the outputs out of, the graph's fixed buffers).  Returns once everything is
         enqueued; out_hosts are valid after a synchronize."""
         main = torch.cuda.current_stream(self.device)
         if not hasattr(self, "_copy_s"):
             self._copy_s = torch.cuda.Stream(self.device)
             self._q2 = [torch.empty(self.out.shape, dtype=torch.bfloat16, device=self.device) for _ in range(2)]
             self._out2 = [torch.empty_like(self.out) for _ in range(2)]
+        if use_graph and resident_scripts is not None:
+            raise ValueError("steps that reset the tables from a script are not captured")
+        if use_graph:
+            self.prepare_host_graph()
         cp = self._copy_s
         n = len(q_hosts)
         ev_up = [torch.cuda.Event() for _ in range(n)]
@@ -411,8 +423,13 @@ class DecodeSession:
             main.wait_event(ev_up[i])
             if i >= 2:
                 main.wait_event(ev_down[i - 2])              # the download that last read this output buffer
-            self.decode_step(self._q2[i % 2], overlapped=True, out=self._out2[i % 2],
-                             resident_script=None if resident_scripts is None else resident_scripts[i])
+            if use_graph:
+                self._q_static.copy_(self._q2[i % 2], non_blocking=True)
+                self.replay_step(self._host_graph)
+                self._out2[i % 2].copy_(self.out, non_blocking=True)
+            else:
+                self.decode_step(self._q2[i % 2], overlapped=True, out=self._out2[i % 2],
+                                 resident_script=None if resident_scripts is None else resident_scripts[i])
             ev_done[i].record(main)
             with torch.cuda.stream(cp):
                 cp.wait_event(ev_done[i])

@@ -402,7 +402,7 @@ def test_double_buffered_host_stepping_matches_plain_stepping():
     cfg = tiny_config(batch=3, ctx=2048, n_q_heads=16, n_kv_heads=4, budget_blocks=24, resident_frac=0.3, n_layers=3)
     steps = 5
     outs = []
-    for form in ("plain", "host"):
+    for form in ("plain", "host", "host+graph"):
         pi = PulseInfer.from_workload(cfg)
         sess = DecodeSession(pi, cfg.batch, cfg.n_layers)
         sess.ctx_len.fill_(cfg.ctx)
@@ -419,7 +419,7 @@ def test_double_buffered_host_stepping_matches_plain_stepping():
         else:
             q_host = q_all.cpu().pin_memory()
             out_host = [torch.empty(sess.out.shape, dtype=torch.bfloat16, pin_memory=True) for _ in range(steps)]
-            sess.decode_steps_from_host([q_host[t] for t in range(steps)], out_host)
+            sess.decode_steps_from_host([q_host[t] for t in range(steps)], out_host, use_graph=form == "host+graph")
             torch.cuda.synchronize()
             got = [o.clone() for o in out_host]
         assert pi.status()[0] == 0
@@ -427,6 +427,7 @@ def test_double_buffered_host_stepping_matches_plain_stepping():
         pi.close()
     for t in range(steps):
         assert torch.equal(outs[0][t].view(torch.int16), outs[1][t].view(torch.int16)), f"step {t}"
+        assert torch.equal(outs[0][t].view(torch.int16), outs[2][t].view(torch.int16)), f"step {t}, graph replay"
 
 
 def test_headwise_attention_with_unequal_and_empty_head_lists():
