@@ -236,7 +236,8 @@ int pi_append_kv(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* k
  * sequence s is page page_table_dev[s * page_table_seq_stride + u] (int32, device memory).  The
  * extents still name logical units; each 4 KB piece looks its page up, so merged extents need no
  * physical adjacency.  All other arguments as in pi_recall_gather_scatter / pi_append_kv; a page
- * index outside [0, n_pages) sets PI_ERR_INDEX_RANGE in the status word and the unit is skipped.
+ * index outside [0, n_pages), or a unit index beyond the sequence's table row (page_table_seq_stride
+ * entries, >= 1), sets PI_ERR_INDEX_RANGE in the status word and the unit is skipped.
  * The caller owns the page table and must have assigned the page of a block before the append
  * that opens it. */
 int pi_recall_gather_scatter_paged(pi_ctx* ctx, int layer, int n_lists, int lists_per_seq,

@@ -228,7 +228,7 @@ extern "C" int pi_recall_gather_scatter_paged(pi_ctx* ctx, int layer, int n_list
                                               int32_t list_capacity, const int32_t* recall_count_dev,
                                               int64_t unit_bytes, int64_t unit_stride_bytes,
                                               int64_t list_offset_bytes, void* stream) {
-    if (!page_table_dev || page_table_seq_stride < 0 || n_pages < 1) return PI_ERR_INVALID_ARG;
+    if (!page_table_dev || page_table_seq_stride < 1 || n_pages < 1) return PI_ERR_INVALID_ARG;
     return recall_call(ctx, layer, n_lists, lists_per_seq, host_arena_pinned, 0, page_table_dev, page_table_seq_stride,
                        n_pages, pool_dev, pool_seq_stride_bytes, recall_list_dev, list_capacity, recall_count_dev,
                        unit_bytes, unit_stride_bytes, list_offset_bytes, stream);
@@ -305,7 +305,7 @@ extern "C" int pi_append_kv_paged(pi_ctx* ctx, int layer, int batch, uint32_t st
                                   const int32_t* page_table_dev, int64_t page_table_seq_stride, int32_t n_pages,
                                   void* pool_dev, int32_t* block_table_dev, int32_t* slot_block_dev,
                                   uint32_t* slot_stamp_dev, void* digest_dev, void* stream) {
-    if (!page_table_dev || page_table_seq_stride < 0 || n_pages < 1) return PI_ERR_INVALID_ARG;
+    if (!page_table_dev || page_table_seq_stride < 1 || n_pages < 1) return PI_ERR_INVALID_ARG;
     return append_call(ctx, layer, batch, step, k_new_dev, v_new_dev, ctx_len_dev, host_arena_pinned, 0,
                        page_table_dev, page_table_seq_stride, n_pages, pool_dev, block_table_dev, slot_block_dev,
                        slot_stamp_dev, digest_dev, stream);

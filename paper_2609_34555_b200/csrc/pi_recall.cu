@@ -165,7 +165,9 @@ recall_kernel(RecallParams p) {
         const long long loff = (l - seq * p.lists_per_seq) * p.list_offset + in_unit + lane * 16;
         if (PAGED) {
             // one table lookup per 4 KB piece; the pieces of a page stay one sequential burst
-            const int pg = p.page[seq * p.page_stride + e.src_unit + k];
+            // a unit index beyond the sequence's row of the table is not followed (rows are page_stride long)
+            const long long ui = static_cast<long long>(e.src_unit) + k;
+            const int pg = ui < p.page_stride ? p.page[seq * p.page_stride + ui] : -1;
             if (pg < 0 || pg >= p.n_pages) {
                 if (lane == 0) pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_RECALL, l, e.src_unit + k, pg);
                 return;

@@ -235,6 +235,9 @@ class DecodeSession:
         self._ev_start = torch.cuda.Event()
         self._path = RecallPath(pi)
         self.step_count = 0
+        self._copy_s = None                  # copy stream and double buffers of the end-to-end form (made on first use)
+        self._host_graph = None
+        self._step_dev_shadow = None
 
     def host_region(self, layer: int) -> torch.Tensor:
         """The layer's host store: [batch][NB] blocks in block order, or (paged) the arena of pages."""
@@ -371,7 +374,7 @@ class DecodeSession:
 
     def replay_step(self, graph: "torch.cuda.CUDAGraph") -> None:
         """One decode step by replaying a graph from capture_step on the current stream."""
-        if getattr(self, "_step_dev_shadow", None) != self.step_count:
+        if self._step_dev_shadow != self.step_count:
             self.step_dev.fill_(self.step_count)          # eager steps ran in between: resynchronise the device counter
         self.step_count += 1
         self._step_dev_shadow = self.step_count           # the replay adds one on the device
@@ -379,7 +382,7 @@ class DecodeSession:
 
     def prepare_host_graph(self) -> None:
         """Captures the graph decode_steps_from_host(use_graph=True) replays (synchronises; once)."""
-        if getattr(self, "_host_graph", None) is None:
+        if self._host_graph is None:
             self._q_static = torch.empty(self.out.shape, dtype=torch.bfloat16, device=self.device)
             self._host_graph = self.capture_step(self._q_static)
 
@@ -392,7 +395,7 @@ class DecodeSession:
         into, and the outputs out of, the graph's fixed buffers).  Returns once everything is
         enqueued; out_hosts are valid after a synchronize."""
         main = torch.cuda.current_stream(self.device)
-        if not hasattr(self, "_copy_s"):
+        if self._copy_s is None:
             self._copy_s = torch.cuda.Stream(self.device)
             self._q2 = [torch.empty(self.out.shape, dtype=torch.bfloat16, device=self.device) for _ in range(2)]
             self._out2 = [torch.empty_like(self.out) for _ in range(2)]
