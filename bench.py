@@ -225,7 +225,7 @@ def run_ours(args) -> dict:
     n_e2e = K if not args.no_e2e else 0
     n_serial = min(K, 4)
     n_graph = min(K, 16) if (not args.append and not args.no_graph) else 0
-    total_steps = args.settle + W + K + 2 * n_serial + n_e2e + n_graph + 1
+    total_steps = args.settle + W + K + 3 * n_serial + n_e2e + n_graph + 1
     pi, sess, R = build_session(cfg, rank, args.host_layers, world, args.recall_ctas,
                                 ctx_start=cfg.ctx - total_steps - 1 if args.append else 0, paged=args.paged,
                                 recall_streams=args.recall_streams, attn_ctas=args.attn_ctas)
@@ -274,8 +274,15 @@ def run_ours(args) -> dict:
     # settling steps (workload preparation, not warm-up): the hot set starts as a uniform
     # draw, so the first steps recall far more than the steady state does
     t = 0
-    for _ in range(args.settle):
+    cold = None
+    for i in range(args.settle):
+        if i == 0:
+            pi.stats(reset=True)
         sess.decode_step(q_all[t], resident_script=script(t), new_kv=new_kv); t += 1
+        if i == 0:                                         # the cold first step, reported apart
+            torch.cuda.synchronize()
+            st0 = pi.stats(reset=True)
+            cold = st0["missing_blocks"] / max(1, st0["sequences"])
     for _ in range(W):
         sess.decode_step(q_all[t], resident_script=script(t), new_kv=new_kv); t += 1
     barrier()
@@ -321,6 +328,22 @@ def run_ours(args) -> dict:
     serial_ms = s0.elapsed_time(s1) / max(1, n_serial)
     ser_stats = pi.stats(reset=True)
     ser = ser_timer.summary()
+
+    # ---------------- distribution of the miss counts: a few more steps, read back after each
+    # (per sequence and layer-step: units of the recall lists)
+    hist_edges = [0, 1, 3, 5, 9, 17, 33, 65, 1 << 30]
+    hist = [0] * (len(hist_edges) - 1)
+    for _ in range(n_serial):
+        sess.decode_step(q_all[t], resident_script=script(t), new_kv=new_kv); t += 1
+        torch.cuda.synchronize()
+        for b in sess.bufs:
+            idx = torch.arange(b.recall_list.shape[1], device=dev)[None, :] < b.recall_count[:, None]
+            per_seq = (b.recall_list[:, :, 2] * idx).sum(dim=1).cpu().numpy()
+            for k in range(len(hist)):
+                hist[k] += int(((per_seq >= hist_edges[k]) & (per_seq < hist_edges[k + 1])).sum())
+    pi.stats(reset=True)
+    miss_hist = {("0" if k == 0 else f"{hist_edges[k]}-{hist_edges[k + 1] - 1}" if k < len(hist) - 1 else f"{hist_edges[k]}+"): hist[k]
+                 for k in range(len(hist))}
 
     # ---------------- the pipelined step captured once into a CUDA graph and replayed (scripted-miss
     # workloads reset their tables from the host every step and stay eager)
@@ -434,6 +457,8 @@ def run_ours(args) -> dict:
                    "pipeline": f"select+diff on stream A, recall pulls rotating over {len(sess.recall_streams)} stream(s), attention on the main stream",
                    "sequence_layer_steps_per_s": world * K * cfg.n_layers * cfg.batch / (ms * 1e-3),
                    "misses_per_seq_layer_step": stats["missing_blocks"] / max(1, stats["sequences"]),
+                   "misses_per_seq_layer_step_cold_first_step": cold,
+                   "miss_histogram_per_seq_layer_step": miss_hist,
                    "miss_script": cfg.miss_script or "none (LRU)", "append": bool(args.append),
                    "settle_steps": args.settle, "setup_s": round(setup_s, 1)},
         "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * n_launch,      # launches inside the timed region only
