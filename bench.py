@@ -536,8 +536,21 @@ def cpu_baseline(cfg, sess, budget_s: float) -> dict:
         el = time.perf_counter() - t0
         if el >= budget_s or step >= 4096:
             break
-    return dict(value=done / el, unit="layer-steps/s", cores=oracle.num_threads(), kind="oracle",
-                sample=f"{done} whole-batch layer-steps (layers {layers}, {step} decode steps) in {el:.1f} s; "
+    cores = oracle.num_threads()
+    # the same on one thread, two layer-steps (context: what the loop over sequences gains)
+    oracle.set_num_threads(1)
+    t1 = time.perf_counter()
+    for l in layers:
+        s = st[l]
+        step += 1
+        r = oracle.layer_step(ctx_len, cfg.n_blocks, cfg.block_tokens, cfg.n_kv_heads, s["h"], cfg.budget_blocks,
+                              cfg.n_sink_blocks, cfg.n_local_blocks, step, q[l][(step - 1) % 64], s["digest"],
+                              s["kvb"], s["table"], s["slot_block"], s["slot_stamp"], s["pool"])
+        assert r["rc"] == 0
+    single = len(layers) / (time.perf_counter() - t1)
+    oracle.set_num_threads(cores)
+    return dict(value=done / el, unit="layer-steps/s", cores=cores, kind="oracle", single_thread_value=single,
+                sample=f"{done} whole-batch layer-steps (layers {layers}, {step - len(layers)} decode steps) in {el:.1f} s; "
                        f"host: {os.cpu_count()} cores")
 
 

@@ -62,6 +62,11 @@ def num_threads() -> int:
     return int(lib().pio_num_threads())
 
 
+def set_num_threads(n: int) -> None:
+    """Threads of the loop over sequences in layer_step (timing only)."""
+    lib().pio_set_num_threads(int(n))
+
+
 def build_digest(kv_seq: np.ndarray, ctx: int, h_star: int) -> np.ndarray:
     """kv_seq uint16 [n_blocks][Hkv][2][B][D] -> digest uint16 [n_blocks][2][D]."""
     nb, Hkv, _, B, D = kv_seq.shape

@@ -48,6 +48,15 @@ int pio_num_threads(void) {
 #endif
 }
 
+/* Threads of the loop over sequences in pio_layer_step (timing only; no effect on results). */
+void pio_set_num_threads(int n) {
+#ifdef _OPENMP
+    if (n >= 1) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 /* Offset (in elements) of token t of kv head h, plane kv (0 = K, 1 = V) in one block
  * stored as [Hkv][2][B][D]. */
 static size_t in_block(int h, int kv, int t, int B, int D) {
