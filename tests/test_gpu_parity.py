@@ -576,3 +576,25 @@ def test_graph_replayed_decode_steps_match_eager_steps():
         assert torch.equal(results[0][0][t].view(torch.int16), results[1][0][t].view(torch.int16)), f"outputs of step {t}"
     for a, b in zip(results[0][1], results[1][1]):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_shapes_of_the_rows_beyond_the_hot_path(seed):
+    """Randomly drawn shapes for the selection strategies with per-head attention (seed % 3 == 0), the
+    append (1) and the pipelined session, with or without append and paging (2)."""
+    from tests.parity import run_append_and_compare, run_session_sampled, run_strategies_and_compare
+    rng = np.random.default_rng(5000 + seed)
+    Hkv, G, B = int(rng.choice([1, 2, 4, 8])), int(rng.choice([1, 2, 4, 8, 16])), int(rng.choice([16, 32, 64]))
+    batch, nb = int(rng.integers(1, 4)), int(rng.integers(40, 120))
+    pinned = 1 + max(1, 128 // B)
+    K = int(rng.integers(pinned + 2, pinned + 24))
+    cfg = tiny_config(batch=batch, ctx=nb * B - int(rng.integers(0, B)), n_q_heads=Hkv * G, n_kv_heads=Hkv, block_tokens=B,
+                      budget_blocks=K, resident_frac=float(rng.uniform(0.4, 0.9)), seed=seed)
+    if seed % 3 == 0:
+        run_strategies_and_compare(cfg, steps=2)
+    elif seed % 3 == 1:
+        lens = [int(rng.integers(cfg.ctx // 2, cfg.ctx - 40)) for _ in range(batch)]
+        run_append_and_compare(cfg, steps=int(rng.integers(5, 40)), ctx_len0=lens)
+    else:
+        run_session_sampled(cfg.replace(n_layers=2), steps=6, sample_seqs=[0], append=bool(seed % 2),
+                            ctx_start=cfg.ctx - 10 if seed % 2 else 0, paged=bool((seed // 2) % 2))
