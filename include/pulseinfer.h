@@ -50,7 +50,7 @@ typedef struct pi_ctx pi_ctx;
 
 typedef struct {
     int32_t n_layers;
-    int32_t n_q_heads, n_kv_heads, head_dim;  /* head_dim must be 128; Hq % Hkv == 0; G <= 16; Hkv <= 16 */
+    int32_t n_q_heads, n_kv_heads, head_dim;  /* head_dim must be 128; Hq % Hkv == 0; G <= 16; Hkv <= 16 (the attention calls: Hkv <= 8) */
     int32_t block_tokens;                     /* 16, 32 or 64                                      */
     int32_t budget_blocks;                    /* K: sink + local + middle blocks per (seq, layer) */
     int32_t n_sink_blocks, n_local_blocks;    /* always-resident, always-selected prefix / suffix */
