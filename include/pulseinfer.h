@@ -252,6 +252,17 @@ int pi_append_kv_paged(pi_ctx* ctx, int layer, int batch, uint32_t step, const v
                        void* pool_dev, int32_t* block_table_dev, int32_t* slot_block_dev,
                        uint32_t* slot_stamp_dev, void* digest_dev, void* stream);
 
+/* pi_append_kv with the step number read from device memory when the kernel runs (see
+ * pi_diff_misses_devstep), for appends inside a replayed CUDA graph.  page_table_dev may be NULL
+ * (block-major store, host_seq_stride_bytes used) or a page table as in pi_append_kv_paged (then
+ * host_kv_pinned is the arena and host_seq_stride_bytes is ignored). */
+int pi_append_kv_devstep(pi_ctx* ctx, int layer, int batch, const uint32_t* step_dev, const void* k_new_dev,
+                         const void* v_new_dev, const int32_t* ctx_len_dev, void* host_kv_pinned,
+                         int64_t host_seq_stride_bytes, const int32_t* page_table_dev,
+                         int64_t page_table_seq_stride, int32_t n_pages, void* pool_dev,
+                         int32_t* block_table_dev, int32_t* slot_block_dev, uint32_t* slot_stamp_dev,
+                         void* digest_dev, void* stream);
+
 /* Helpers around the path (input preparation and measurement; not hot calls).
  * pi_build_digests: channel-wise min / max of the keys of head solo_head[layer] over the
  *   valid tokens of each block; kv may be device memory or pinned host memory laid out

@@ -23,7 +23,7 @@ ERR_NAMES = {
 EXTENT_DTYPE = torch.int32      # a pi_extent is four int32: src_unit, dst_unit, n_units, units_before
 
 EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_score_select_noalloc", "pi_score_select_strategy", "pi_diff_misses", "pi_diff_misses_devstep", "pi_recall_gather_scatter",
-           "pi_recall_gather_scatter_paged", "pi_sparse_decode_attn", "pi_sparse_decode_attn_headwise", "pi_append_kv", "pi_append_kv_paged", "pi_build_digests", "pi_build_digests_all", "pi_table_init", "pi_h2d_copy_ms",
+           "pi_recall_gather_scatter_paged", "pi_sparse_decode_attn", "pi_sparse_decode_attn_headwise", "pi_append_kv", "pi_append_kv_paged", "pi_append_kv_devstep", "pi_build_digests", "pi_build_digests_all", "pi_table_init", "pi_h2d_copy_ms",
            "pi_get_status", "pi_get_stats", "pi_clear_status", "pi_strerror"]
 
 
@@ -65,6 +65,8 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
                                                    c_int32, i32p, c_int64, c_int64, c_int64, vp]
     lib.pi_append_kv_paged.argtypes = [c_void_p, c_int, c_int, c_uint32, vp, vp, i32p, vp, i32p, c_int64, c_int32, vp, i32p,
                                        i32p, u32p, vp, vp]
+    lib.pi_append_kv_devstep.argtypes = [c_void_p, c_int, c_int, u32p, vp, vp, i32p, vp, c_int64, i32p, c_int64, c_int32, vp,
+                                         i32p, i32p, u32p, vp, vp]
     lib.pi_score_select_strategy.argtypes = [c_void_p, c_int, c_int, c_int, vp, vp, i32p, i32p, i32p, vp, vp]
     lib.pi_build_digests_all.argtypes = [c_void_p, c_int, vp, c_int64, i32p, vp, vp]
     lib.pi_sparse_decode_attn.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, i32p, vp, vp, vp]
@@ -269,6 +271,19 @@ class PulseInfer:
         batch = ctx_len.shape[0]
         if not host_kv.is_cuda and not host_kv.is_pinned():
             raise PiError("pi_append_kv", -5, strerror(-5))
+        if isinstance(step, torch.Tensor):               # the step number lives on the device (graph replay)
+            pages = 0
+            if page_table is not None:
+                pages = n_pages if n_pages is not None else host_kv.numel() * host_kv.element_size() // self.block_bytes
+            hs = host_seq_stride if host_seq_stride is not None else host_kv.stride(0) * host_kv.element_size()
+            _check("pi_append_kv_devstep", self._lib.pi_append_kv_devstep(
+                self._ctx, layer, batch, _dev(step, torch.int32, "step"), _dev(k_new, torch.bfloat16, "k_new"),
+                _dev(v_new, torch.bfloat16, "v_new"), _dev(ctx_len, torch.int32, "ctx_len"), host_kv.data_ptr(), hs,
+                None if page_table is None else _dev(page_table, torch.int32, "page_table"),
+                0 if page_table is None else page_table.stride(0), pages, pool.data_ptr(),
+                _dev(block_table, torch.int32, "block_table"), _dev(slot_block, torch.int32, "slot_block"),
+                _dev(slot_stamp, torch.int32, "slot_stamp"), _dev(digest, torch.bfloat16, "digest"), _stream(stream)))
+            return
         if page_table is not None:
             pages = n_pages if n_pages is not None else host_kv.numel() * host_kv.element_size() // self.block_bytes
             _check("pi_append_kv_paged", self._lib.pi_append_kv_paged(

@@ -264,7 +264,7 @@ extern "C" int pi_sparse_decode_attn_headwise(pi_ctx* ctx, int layer, int batch,
                      out_dev, lse_dev, 1, stream);
 }
 
-static int append_call(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* k_new_dev, const void* v_new_dev,
+static int append_call(pi_ctx* ctx, int layer, int batch, uint32_t step, const uint32_t* step_dev, const void* k_new_dev, const void* v_new_dev,
                        const int32_t* ctx_len_dev, void* host_kv_pinned, int64_t host_seq_stride_bytes,
                        const int32_t* page_table, int64_t page_stride, int32_t n_pages, void* pool_dev,
                        int32_t* block_table_dev, int32_t* slot_block_dev, uint32_t* slot_stamp_dev, void* digest_dev,
@@ -272,7 +272,7 @@ static int append_call(pi_ctx* ctx, int layer, int batch, uint32_t step, const v
     int rc = check_call(ctx, layer, batch);
     if (rc != PI_OK) return rc;
     if (!k_new_dev || !v_new_dev || !ctx_len_dev || !host_kv_pinned || !pool_dev || !block_table_dev ||
-        !slot_block_dev || !slot_stamp_dev || !digest_dev || step == 0 || host_seq_stride_bytes < 0)
+        !slot_block_dev || !slot_stamp_dev || !digest_dev || (!step_dev && step == 0) || host_seq_stride_bytes < 0)
         return PI_ERR_INVALID_ARG;
     if (!pi_aligned16(k_new_dev) || !pi_aligned16(v_new_dev) || !pi_aligned16(host_kv_pinned) ||
         !pi_aligned16(pool_dev) || !pi_aligned16(digest_dev) || host_seq_stride_bytes % 16)
@@ -288,14 +288,14 @@ static int append_call(pi_ctx* ctx, int layer, int batch, uint32_t step, const v
     }
     return pi_launch_append(ctx, ctx->solo_head[layer], batch, step, k_new_dev, v_new_dev, ctx_len_dev, dst,
                             host_seq_stride_bytes, pool_dev, block_table_dev, slot_block_dev, slot_stamp_dev,
-                            digest_dev, page_table, page_stride, n_pages, static_cast<cudaStream_t>(stream));
+                            digest_dev, page_table, page_stride, n_pages, step_dev, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int pi_append_kv(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* k_new_dev,
                             const void* v_new_dev, const int32_t* ctx_len_dev, void* host_kv_pinned,
                             int64_t host_seq_stride_bytes, void* pool_dev, int32_t* block_table_dev,
                             int32_t* slot_block_dev, uint32_t* slot_stamp_dev, void* digest_dev, void* stream) {
-    return append_call(ctx, layer, batch, step, k_new_dev, v_new_dev, ctx_len_dev, host_kv_pinned,
+    return append_call(ctx, layer, batch, step, nullptr, k_new_dev, v_new_dev, ctx_len_dev, host_kv_pinned,
                        host_seq_stride_bytes, nullptr, 0, 0, pool_dev, block_table_dev, slot_block_dev,
                        slot_stamp_dev, digest_dev, stream);
 }
@@ -306,9 +306,22 @@ extern "C" int pi_append_kv_paged(pi_ctx* ctx, int layer, int batch, uint32_t st
                                   void* pool_dev, int32_t* block_table_dev, int32_t* slot_block_dev,
                                   uint32_t* slot_stamp_dev, void* digest_dev, void* stream) {
     if (!page_table_dev || page_table_seq_stride < 1 || n_pages < 1) return PI_ERR_INVALID_ARG;
-    return append_call(ctx, layer, batch, step, k_new_dev, v_new_dev, ctx_len_dev, host_arena_pinned, 0,
+    return append_call(ctx, layer, batch, step, nullptr, k_new_dev, v_new_dev, ctx_len_dev, host_arena_pinned, 0,
                        page_table_dev, page_table_seq_stride, n_pages, pool_dev, block_table_dev, slot_block_dev,
                        slot_stamp_dev, digest_dev, stream);
+}
+
+extern "C" int pi_append_kv_devstep(pi_ctx* ctx, int layer, int batch, const uint32_t* step_dev, const void* k_new_dev,
+                                    const void* v_new_dev, const int32_t* ctx_len_dev, void* host_kv_pinned,
+                                    int64_t host_seq_stride_bytes, const int32_t* page_table_dev,
+                                    int64_t page_table_seq_stride, int32_t n_pages, void* pool_dev,
+                                    int32_t* block_table_dev, int32_t* slot_block_dev, uint32_t* slot_stamp_dev,
+                                    void* digest_dev, void* stream) {
+    if (!step_dev) return PI_ERR_INVALID_ARG;
+    if (page_table_dev && (page_table_seq_stride < 1 || n_pages < 1)) return PI_ERR_INVALID_ARG;
+    return append_call(ctx, layer, batch, 0, step_dev, k_new_dev, v_new_dev, ctx_len_dev, host_kv_pinned,
+                       page_table_dev ? 0 : host_seq_stride_bytes, page_table_dev, page_table_seq_stride, n_pages,
+                       pool_dev, block_table_dev, slot_block_dev, slot_stamp_dev, digest_dev, stream);
 }
 
 extern "C" int pi_build_digests(pi_ctx* ctx, int layer, int batch, const void* kv, int64_t kv_seq_stride_bytes,

@@ -24,6 +24,7 @@ struct AppendParams {
     const int32_t* page;           // paged host store (or null): block b of sequence s is arena page page[s * page_stride + b]
     long long page_stride;
     int n_pages;
+    const uint32_t* step_dev;      // when set, the stamp is read from device memory (graph replay)
     uint32_t step;
     int B, Hkv, C, n_sink, n_local, max_blocks, h_star;
 };
@@ -103,7 +104,7 @@ append_kernel(AppendParams p) {
         }
         __syncthreads();                                   // zeros land before the rows below
     }
-    if (tid == 0) slot_stamp[slot] = p.step;
+    if (tid == 0) slot_stamp[slot] = p.step_dev ? *p.step_dev : p.step;
     // rows: [Hkv][2][B][D]; one head row is 256 B = 16 uint4
     for (int i = tid; i < p.Hkv * 32; i += APPEND_THREADS) {
         const int h = i >> 5, kv = (i >> 4) & 1, c = i & 15;
@@ -130,8 +131,9 @@ append_kernel(AppendParams p) {
 int pi_launch_append(pi_ctx* c, int h_star, int batch, uint32_t step, const void* k_new, const void* v_new,
                      const int32_t* ctx_len, void* host_kv, int64_t host_stride, void* pool, int32_t* table,
                      int32_t* slot_block, uint32_t* slot_stamp, void* digest, const int32_t* page_table,
-                     int64_t page_stride, int32_t n_pages, cudaStream_t stream) {
+                     int64_t page_stride, int32_t n_pages, const uint32_t* step_dev, cudaStream_t stream) {
     AppendParams p;
+    p.step_dev = step_dev;
     p.page = page_table; p.page_stride = page_stride; p.n_pages = n_pages;
     p.k_new = static_cast<const uint4*>(k_new);
     p.v_new = static_cast<const uint4*>(v_new);

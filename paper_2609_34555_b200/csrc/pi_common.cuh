@@ -93,7 +93,7 @@ int pi_launch_attn(pi_ctx*, int batch, const void* q, const void* pool, const in
 int pi_launch_append(pi_ctx*, int h_star, int batch, uint32_t step, const void* k_new, const void* v_new,
                      const int32_t* ctx_len, void* host_kv, int64_t host_stride, void* pool, int32_t* table,
                      int32_t* slot_block, uint32_t* slot_stamp, void* digest, const int32_t* page_table,
-                     int64_t page_stride, int32_t n_pages, cudaStream_t);
+                     int64_t page_stride, int32_t n_pages, const uint32_t* step_dev, cudaStream_t);
 int pi_launch_build_digests_all(pi_ctx*, int batch, const void* kv, int64_t stride, const int32_t* ctx_len,
                                 void* digest_all, cudaStream_t);
 int pi_launch_build_digests(pi_ctx*, int h_star, int batch, const void* kv, int64_t stride,

@@ -358,16 +358,19 @@ class DecodeSession:
                 if t4 is not None: tm.add("attn", t4, t5)
         return out
 
-    def capture_step(self, q_static: torch.Tensor, out: Optional[torch.Tensor] = None) -> "torch.cuda.CUDAGraph":
+    def capture_step(self, q_static: torch.Tensor, out: Optional[torch.Tensor] = None,
+                     new_kv_static=None) -> "torch.cuda.CUDAGraph":
         """Captures one pipelined decode step (all layers, all streams) into a CUDA graph that reads
         its queries from `q_static` and its step number from device memory.  Replays continue the
-        session: call `graph.replay()` once per decode step after refreshing `q_static` (stream
-        order serialises consecutive replays, as consecutive decode steps are anyway).  Eager steps
-        and replays may be mixed; steps that append tokens or reset the tables stay eager."""
+        session: call `replay_step(graph)` once per decode step after refreshing `q_static` (stream
+        order serialises consecutive replays, as consecutive decode steps are anyway).  With
+        new_kv_static = (k, v) buffers the graph also appends the step's token (refresh them too;
+        the context lengths advance on the device).  Eager steps and replays may be mixed; steps
+        that reset the tables from a script stay eager."""
         torch.cuda.synchronize(self.device)
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
-            self.decode_step(q_static, overlapped=True, out=out, capturing=True)
+            self.decode_step(q_static, overlapped=True, out=out, capturing=True, new_kv=new_kv_static)
         self.step_count -= 1                              # the capture itself ran nothing
         self._step_dev_shadow = None
         return graph

@@ -598,3 +598,57 @@ def test_random_shapes_of_the_rows_beyond_the_hot_path(seed):
     else:
         run_session_sampled(cfg.replace(n_layers=2), steps=6, sample_seqs=[0], append=bool(seed % 2),
                             ctx_start=cfg.ctx - 10 if seed % 2 else 0, paged=bool((seed // 2) % 2))
+
+
+def test_graph_replay_with_append_matches_eager_steps():
+    """The captured step also appends the step's token (stamp and context length from device memory):
+    outputs, context lengths, digests, tables and the host store equal those of eager stepping."""
+    import torch
+    from paper_2609_34555_b200 import PulseInfer
+    from paper_2609_34555_b200.runner import DecodeSession
+    from workloads import generate as gen
+    cfg = tiny_config(batch=3, ctx=2048, n_q_heads=16, n_kv_heads=4, budget_blocks=24, resident_frac=0.3, n_layers=2)
+    steps, ctx0 = 8, 2048 - 21                              # the context crosses a block boundary (2032) at step 6
+    results = []
+    for form in ("eager", "graph"):
+        pi = PulseInfer.from_workload(cfg)
+        sess = DecodeSession(pi, cfg.batch, cfg.n_layers)
+        sess.ctx_len.fill_(ctx0)
+        short = cfg.replace(ctx=ctx0)
+        for l in range(cfg.n_layers):
+            kv = gen.make_kv(cfg, l, device=sess.device)
+            sess.load_layer(l, kv, torch.from_numpy(gen.initial_resident(short, l)).to(sess.device))
+        q_all = torch.stack([gen.make_queries(cfg, l, steps, device=sess.device) for l in range(cfg.n_layers)], 1).contiguous()
+        g = torch.Generator(device=sess.device).manual_seed(77)
+        shp = (steps, cfg.n_layers, cfg.batch, cfg.n_kv_heads, cfg.head_dim)
+        k_all = torch.randn(shp, device=sess.device, generator=g).to(torch.bfloat16)
+        v_all = torch.randn(shp, device=sess.device, generator=g).to(torch.bfloat16)
+        got = []
+        if form == "eager":
+            for t in range(steps):
+                sess.decode_step(q_all[t], new_kv=(k_all[t], v_all[t]))
+                torch.cuda.synchronize()
+                got.append(sess.out.cpu().clone())
+        else:
+            sess.decode_step(q_all[0], new_kv=(k_all[0], v_all[0]))
+            torch.cuda.synchronize()
+            got.append(sess.out.cpu().clone())
+            q_s, k_s, v_s = q_all[0].clone(), k_all[0].clone(), v_all[0].clone()
+            graph = sess.capture_step(q_s, new_kv_static=(k_s, v_s))
+            for t in range(1, steps):
+                q_s.copy_(q_all[t]); k_s.copy_(k_all[t]); v_s.copy_(v_all[t])
+                sess.replay_step(graph)
+                torch.cuda.synchronize()
+                got.append(sess.out.cpu().clone())
+        assert pi.status()[0] == 0, pi.status()
+        state = [sess.ctx_len.cpu()] + [torch.stack([getattr(b, name).cpu() for b in sess.bufs])
+                                         for name in ("block_table", "slot_stamp", "sel_slots")]
+        state += [torch.stack([b.digest.cpu().view(torch.int16) for b in sess.bufs]),
+                  torch.stack([sess.host_region(l).view(torch.int16).clone() for l in range(cfg.n_layers)])]
+        results.append((got, state))
+        pi.close()
+    assert int(results[0][1][0][0]) == ctx0 + steps
+    for t in range(steps):
+        assert torch.equal(results[0][0][t].view(torch.int16), results[1][0][t].view(torch.int16)), f"outputs of step {t}"
+    for a, b in zip(results[0][1], results[1][1]):
+        assert torch.equal(a, b)
