@@ -224,7 +224,7 @@ def run_ours(args) -> dict:
     t_setup = time.time()
     n_e2e = K if not args.no_e2e else 0
     n_serial = min(K, 4)
-    n_graph = min(K, 16) if (not args.append and not args.no_graph) else 0
+    n_graph = min(K, 16) if not args.no_graph else 0
     total_steps = args.settle + W + K + 3 * n_serial + n_e2e + n_graph + 1
     pi, sess, R = build_session(cfg, rank, args.host_layers, world, args.recall_ctas,
                                 ctx_start=cfg.ctx - total_steps - 1 if args.append else 0, paged=args.paged,
@@ -350,7 +350,7 @@ def run_ours(args) -> dict:
     graph_leg = None
     if n_graph and scripts is None:
         q_static = q_all[t].clone()
-        graph = sess.capture_step(q_static)
+        graph = sess.capture_step(q_static, new_kv_static=new_kv)
         q_static.copy_(q_all[t]); sess.replay_step(graph); t += 1          # one untimed replay
         barrier()
         pi.stats(reset=True)
@@ -403,7 +403,7 @@ def run_ours(args) -> dict:
     if n_e2e:
         q_host = q_all[t:t + n_e2e].cpu().pin_memory()
         out_host = [torch.empty(sess.out.shape, dtype=torch.bfloat16, pin_memory=True) for _ in range(2)]
-        e2e_graph = bool(n_graph) and scripts is None
+        e2e_graph = bool(n_graph) and scripts is None and not args.append
         if e2e_graph:
             sess.prepare_host_graph()                     # capture outside the timed region
         barrier()
