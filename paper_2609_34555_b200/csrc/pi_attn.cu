@@ -5,7 +5,7 @@
 // A persistent grid splits the list evenly (split-K across CTAs, ranges may cross
 // sequence boundaries); a CTA is one TMA producer warp plus one consumer warp per kv
 // head.  The producer streams units through a ring of shared-memory stages with
-// tiled TMA loads (128-byte swizzle, no multicast); consumer warp h computes, for its
+// tiled TMA loads (128-byte swizzle, every CTA fetches its own tiles); consumer warp h computes, for its
 // G query heads,  S^T = K q^T  (tokens on M, heads on N, bf16 mma, fp32 accumulate),
 // an online softmax over tokens, and  O^T += V^T P.  A (CTA, sequence) segment that
 // does not cover its whole sequence writes an fp32 partial (m, l, O); a small second
