@@ -87,6 +87,15 @@ def test_full_size_config4_shapes_group_of_eight_sampled():
     run_session_sampled(cfg, steps=2, sample_seqs=[1, 6])
 
 
+def test_full_size_config3_shapes_block_32_sampled():
+    """Per-sequence shapes of the long-context config (131072 tokens, 4096 blocks of 32 tokens, K 64,
+    C 409) on one layer and 8 of its 64 sequences; the oracle follows two of them."""
+    from tests.parity import run_session_sampled
+    cfg = get_config("c3").replace(n_layers=1, batch=8)
+    stats = run_session_sampled(cfg, steps=3, sample_seqs=[2, 6])
+    assert stats["misses"] > 0
+
+
 def gen_pinned(cfg):
     from workloads import generate as gen
     return gen.pinned_blocks(cfg).tolist()
