@@ -251,9 +251,10 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + ATTN_MAX_STAGES);
     const int SUB = p.B >> 4;
     if (tid == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&pool_map) : "memory");
+    pi_grid_dependency_wait();
     // the merge kernel that follows in the stream may be scheduled from now on; it waits for this
     // grid to finish before it reads anything this grid writes
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    pi_launch_dependents();
 
     // ---- unit prefix over sequences (every CTA computes the same table)
     for (int s = tid; s < p.batch; s += blockDim.x) {
@@ -578,7 +579,7 @@ int pi_launch_attn(pi_ctx* c, int batch, const void* q, const void* pool, const 
     const int threads = (cfg.n_kv_heads + 1) * 32;
     auto launch = [&](auto kernel) -> int {
         PI_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-        kernel<<<c->attn_ctas, threads, smem, stream>>>(c->pool_map, p);
+        PI_CUDA_TRY(pi_launch_pdl(kernel, dim3(c->attn_ctas), dim3(threads), smem, stream, c->pool_map, p));
         return PI_OK;
     };
     int rc;

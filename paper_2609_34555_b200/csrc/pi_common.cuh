@@ -14,6 +14,35 @@
 #define PI_STAGE_ATTN   4
 #define PI_STAGE_APPEND 5
 
+// Programmatic dependent launch.  Every kernel of the path is launched with programmatic stream
+// serialization: its grid may be scheduled while the kernel before it in the stream is still
+// running, which takes the launch latency off the chain select -> diff -> recall -> attention ->
+// merge.  The rule that keeps this safe: a kernel calls pi_grid_dependency_wait() before it reads or
+// writes any global memory (the wait returns once the previous kernel has completed and flushed; it
+// is a no-op after a plain launch), and lets its own dependents in only AFTER that wait, so at most
+// one kernel runs ahead and whatever a kernel reads before its wait was written at least two
+// kernels upstream.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pi_grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pi_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t pi_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                 Args&&... args) {
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = grid;
+    lc.blockDim = block;
+    lc.dynamicSmemBytes = smem;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    return cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 #define PI_HEAD_DIM 128
 #define PI_SELECT_BINS 2048
 

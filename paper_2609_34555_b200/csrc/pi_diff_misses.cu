@@ -58,6 +58,8 @@ __device__ __forceinline__ int ordered_pos(bool flag, int& base, int* warp_tot) 
 __global__ void __launch_bounds__(DIFF_THREADS)
 diff_kernel(DiffParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    pi_grid_dependency_wait();
+    pi_launch_dependents();
     const uint32_t step = p.step_dev ? *p.step_dev : p.step;
     unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);       // [Cpad]
     int32_t* s_sel = reinterpret_cast<int32_t*>(keys + p.Cpad);                         // [K]
@@ -267,7 +269,7 @@ int pi_launch_diff(pi_ctx* c, int batch, uint32_t step, const uint32_t* step_dev
     const size_t smem = static_cast<size_t>(cpad) * 8 + static_cast<size_t>(p.K) * 12 + static_cast<size_t>(p.C);
     if (smem > 40 * 1024)
         PI_CUDA_TRY(cudaFuncSetAttribute(diff_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    diff_kernel<<<batch, DIFF_THREADS, smem, stream>>>(p);
+    PI_CUDA_TRY(pi_launch_pdl(diff_kernel, dim3(batch), dim3(DIFF_THREADS), smem, stream, p));
     PI_CUDA_TRY(cudaGetLastError());
     return PI_OK;
 }

@@ -76,6 +76,8 @@ recall_kernel(RecallParams p) {
     pi_extent* s_ext = reinterpret_cast<pi_extent*>(s_pref + p.n_lists + 1 + (p.n_lists + 2) / 2);   // [cache_cap]
     __shared__ long long warp_tot[RECALL_WARPS];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pi_grid_dependency_wait();
+    pi_launch_dependents();
 
     // 1. extents before each list (counts are validated once, here)
     long long run = 0;
@@ -232,7 +234,7 @@ int pi_launch_recall(pi_ctx* c, int n_lists, int lists_per_seq, const void* host
     // this one needs nearly all of it -- with the default split its CTAs could not join ours
     PI_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                      cudaSharedmemCarveoutMaxShared));
-    kernel<<<c->recall_ctas, RECALL_THREADS, smem, stream>>>(p);
+    PI_CUDA_TRY(pi_launch_pdl(kernel, dim3(c->recall_ctas), dim3(RECALL_THREADS), smem, stream, p));
     PI_CUDA_TRY(cudaGetLastError());
     return PI_OK;
 }

@@ -271,6 +271,8 @@ score_select_kernel(SelParams p) {
     __shared__ int sh_last;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pi_grid_dependency_wait();
+    pi_launch_dependents();
     const int n_chunks = (p.max_blocks + SCORE_CHUNK - 1) / SCORE_CHUNK;
     const int total = n_chunks * p.batch;
     const int f1 = min((static_cast<int>(blockIdx.x) + 1) * p.per, total);
@@ -457,6 +459,8 @@ static int launch_score_select(SelParams& p, int batch, int n_sms, cudaStream_t 
     auto kern = multi ? score_select_kernel<true> : score_select_kernel<false>;
     if (smem > 40 * 1024)
         PI_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    // a plain launch: this grid fills every SM's registers, so it must not sit resident waiting for
+    // the kernel before it (it would keep the attention kernel of the other stream off the SMs)
     kern<<<grid, SCORE_THREADS, smem, stream>>>(p);
     PI_CUDA_TRY(cudaGetLastError());
     return PI_OK;
