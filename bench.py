@@ -225,7 +225,7 @@ def run_ours(args) -> dict:
     n_e2e = K if not args.no_e2e else 0
     n_serial = min(K, 4)
     n_graph = min(K, 16) if not args.no_graph else 0
-    total_steps = args.settle + W + K + 3 * n_serial + n_e2e + n_graph + 1
+    total_steps = args.settle + W + K + 4 * n_serial + n_e2e + n_graph + 1
     pi, sess, R = build_session(cfg, rank, args.host_layers, world, args.recall_ctas,
                                 ctx_start=cfg.ctx - total_steps - 1 if args.append else 0, paged=args.paged,
                                 recall_streams=args.recall_streams, attn_ctas=args.attn_ctas)
@@ -328,6 +328,16 @@ def run_ours(args) -> dict:
     serial_ms = s0.elapsed_time(s1) / max(1, n_serial)
     ser_stats = pi.stats(reset=True)
     ser = ser_timer.summary()
+    # the same chain without events between the calls (events keep the dependent launches of the chain
+    # from overlapping their predecessors)
+    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    p0.record()
+    for _ in range(n_serial):
+        sess.decode_step(q_all[t], overlapped=False, resident_script=script(t), new_kv=new_kv); t += 1
+    p1.record()
+    torch.cuda.synchronize()
+    serial_plain_ms = p0.elapsed_time(p1) / max(1, n_serial)
+    pi.stats(reset=True)
 
     # ---------------- distribution of the miss counts: a few more steps, read back after each
     # (per sequence and layer-step: units of the recall lists)
@@ -484,6 +494,7 @@ def run_ours(args) -> dict:
         "stages_us_events_around_every_call": {k: v["mean_ms"] * 1e3 for k, v in det.items() if v["launches"]},
         "graph_replay": graph_leg,
         "serial": {"layer_steps_per_s": cfg.n_layers / (serial_ms * 1e-3),
+                   "layer_steps_per_s_without_events": cfg.n_layers / (serial_plain_ms * 1e-3),
                    "stages_us": {k: v["mean_ms"] * 1e3 for k, v in ser.items() if v["launches"]}},
         "h2d_peak_gbs": h2d_gbs,
     }
