@@ -34,6 +34,8 @@ append_kernel(AppendParams p) {
     __shared__ unsigned long long warp_min[APPEND_WARPS];
     __shared__ int s_slot;
     const int seq = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pi_grid_dependency_wait();
+    pi_launch_dependents();
     const int pos = p.ctx_len[seq];
     if (pos < 0) return;
     const int b = pos / p.B, t = pos - b * p.B;
@@ -149,7 +151,7 @@ int pi_launch_append(pi_ctx* c, int h_star, int batch, uint32_t step, const void
     p.B = c->cfg.block_tokens; p.Hkv = c->cfg.n_kv_heads; p.C = c->cfg.pool_slots;
     p.n_sink = c->cfg.n_sink_blocks; p.n_local = c->cfg.n_local_blocks; p.max_blocks = c->cfg.max_blocks;
     p.h_star = h_star;
-    append_kernel<<<batch, APPEND_THREADS, 0, stream>>>(p);
+    PI_CUDA_TRY(pi_launch_pdl(append_kernel, dim3(batch), dim3(APPEND_THREADS), 0, stream, p));
     PI_CUDA_TRY(cudaGetLastError());
     return PI_OK;
 }
