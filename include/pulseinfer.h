@@ -50,7 +50,7 @@ typedef struct pi_ctx pi_ctx;
 
 typedef struct {
     int32_t n_layers;
-    int32_t n_q_heads, n_kv_heads, head_dim;  /* head_dim must be 128; Hq % Hkv == 0; G <= 16; Hkv <= 16 (the attention calls: Hkv <= 8) */
+    int32_t n_q_heads, n_kv_heads, head_dim;  /* head_dim must be 128; Hkv a power of two <= 16 (the attention calls: <= 8); Hq % Hkv == 0; G <= 16 */
     int32_t block_tokens;                     /* 16, 32 or 64                                      */
     int32_t budget_blocks;                    /* K: sink + local + middle blocks per (seq, layer) */
     int32_t n_sink_blocks, n_local_blocks;    /* always-resident, always-selected prefix / suffix */
@@ -129,8 +129,8 @@ int pi_score_select_noalloc(int batch, int n_q_heads, int n_kv_heads, int block_
  * Per-head selections go through pi_diff_misses with batch*Hkv rows (tables, slot arrays and a
  * ctx_len array of that many rows) and through pi_recall_gather_scatter with lists_per_seq = Hkv,
  * unit_bytes = frag_bytes, unit_stride_bytes = block_bytes, list_offset_bytes = frag_bytes: head h
- * of slot s then holds the fragment of whatever block head h selected.  Attention over per-head
- * selections is not provided. */
+ * of slot s then holds the fragment of whatever block head h selected; attention over such
+ * per-head selections is pi_sparse_decode_attn_headwise. */
 #define PI_SELECT_AVERAGE  1
 #define PI_SELECT_HEADWISE 2
 int pi_score_select_strategy(pi_ctx* ctx, int strategy, int layer, int batch, const void* q_dev,
@@ -175,6 +175,9 @@ int pi_diff_misses_devstep(pi_ctx* ctx, int layer, int batch, const uint32_t* st
  *   pool_dev                 sequence s starts at pool_dev + s*pool_seq_stride_bytes
  *   recall_list_dev          [n_lists][list_capacity] pi_extent; recall_count_dev [n_lists]
  *   unit_bytes               multiple of 4096
+ *                            An extent whose units reach beyond the sequence's pool region (C blocks) or,
+ *                            in the block-major store, its host region (NB blocks) sets PI_ERR_INDEX_RANGE
+ *                            in the status word (stage 3: list, extent, unit); those units are skipped.
  *   unit_stride_bytes        distance between consecutive units (0 = unit_bytes: units are contiguous)
  *   list_offset_bytes        list i starts (i % lists_per_seq) * list_offset_bytes into its sequence's
  *                            region, in the host store and in the pool alike (0 for the shared selection) */
@@ -224,7 +227,9 @@ int pi_sparse_decode_attn_headwise(pi_ctx* ctx, int layer, int batch, const void
  *   - the slot's stamp becomes `step`.
  *   k_new_dev, v_new_dev  [batch][Hkv][D] bf16;  digest_dev [batch][NB][2][D];  other arrays as in
  *   pi_diff_misses.  Device-side problems (block index beyond NB, nothing evictable, a block that
- *   must be resident is not) set the status word with stage 5 and leave the sequence untouched. */
+ *   must be resident is not) set the status word with stage 5 and leave the sequence untouched.
+ *   Needs n_local_blocks >= 1 (else PI_ERR_INVALID_ARG): the local window is what keeps the block
+ *   that is being filled resident between two appends. */
 int pi_append_kv(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* k_new_dev,
                  const void* v_new_dev, const int32_t* ctx_len_dev, void* host_kv_pinned,
                  int64_t host_seq_stride_bytes, void* pool_dev, int32_t* block_table_dev,

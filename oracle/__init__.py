@@ -34,10 +34,23 @@ def build(force: bool = False) -> Path:
 _lib = None
 
 
+def build_sanitized() -> Path:
+    """The same source with AddressSanitizer and UndefinedBehaviorSanitizer (a test loads it in a
+    child process through PI_ORACLE_LIB, with the sanitizer runtime preloaded)."""
+    out = _HERE / "libpi_oracle_asan.so"
+    if not out.exists() or out.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = out.with_suffix(f".tmp{os.getpid()}.so")
+        subprocess.check_call(["gcc", "-O1", "-g", "-std=c11", "-fopenmp", "-fsanitize=address,undefined",
+                               "-fno-sanitize-recover=undefined", "-fno-omit-frame-pointer", "-shared", "-fPIC",
+                               "-o", str(tmp), str(_SRC), "-lm"])
+        os.replace(tmp, out)
+    return out
+
+
 def lib():
     global _lib
     if _lib is None:
-        _lib = ctypes.CDLL(str(build()))
+        _lib = ctypes.CDLL(os.environ.get("PI_ORACLE_LIB") or str(build()))
         _lib.pio_num_threads.restype = ctypes.c_int
     return _lib
 

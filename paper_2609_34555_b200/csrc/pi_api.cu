@@ -271,6 +271,9 @@ static int append_call(pi_ctx* ctx, int layer, int batch, uint32_t step, const u
                        void* stream) {
     int rc = check_call(ctx, layer, batch);
     if (rc != PI_OK) return rc;
+    // without a local window nothing keeps the block that is being filled resident: a later token of
+    // the same block could find it evicted and be lost from the host store as well
+    if (ctx->cfg.n_local_blocks < 1) return PI_ERR_INVALID_ARG;
     if (!k_new_dev || !v_new_dev || !ctx_len_dev || !host_kv_pinned || !pool_dev || !block_table_dev ||
         !slot_block_dev || !slot_stamp_dev || !digest_dev || (!step_dev && step == 0) || host_seq_stride_bytes < 0)
         return PI_ERR_INVALID_ARG;

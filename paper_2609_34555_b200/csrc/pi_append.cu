@@ -50,7 +50,8 @@ append_kernel(AppendParams p) {
     int slot = table[b];
     long long host_off = seq * p.host_stride + b * block_bytes;
     if (p.page) {
-        const int pg = p.page[seq * p.page_stride + b];
+        // a block index beyond the sequence's row of the table is not followed (rows are page_stride long)
+        const int pg = b < p.page_stride ? p.page[seq * p.page_stride + b] : -1;
         if (pg < 0 || pg >= p.n_pages) {
             if (tid == 0) pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_APPEND, seq, b, pg);
             return;

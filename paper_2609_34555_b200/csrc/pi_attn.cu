@@ -161,13 +161,17 @@ attn_merge_kernel(AttnParams p, int main_ctas) {
     __syncthreads();
     before = mine = total = 0;
     for (int w = 0; w < n_warps; ++w) { before += s_red[0][w]; mine += s_red[1][w]; total += s_red[2][w]; }
-    if (mine == 0) return;                                    // nothing selected: the main kernel wrote zeros
     const long long U = total, P = min(static_cast<long long>(main_ctas), max(U, 1ll));
-    const int c_first = cta_of_unit(before, U, P), c_last = cta_of_unit(before + mine - 1, U, P);
-    const int n_seg = c_last - c_first + 1;
+    int c_first = 0, n_seg = 0;
+    if (mine > 0) {
+        c_first = cta_of_unit(before, U, P);
+        n_seg = cta_of_unit(before + mine - 1, U, P) - c_first + 1;
+    }
+    // Every CTA executes the wait, also the ones with nothing to merge: a dependent grid that retired
+    // without waiting would let the stream move on while the main grid is still writing.
+    pi_grid_dependency_wait();                                // main grid complete, its stores visible
+    if (mine == 0) return;                                    // nothing selected: the main kernel wrote zeros
     if (n_seg == 1) return;                                   // one CTA covered the sequence and wrote the result
-
-    asm volatile("griddepcontrol.wait;" ::: "memory");        // main grid complete, its stores visible
 
     const size_t slot0 = static_cast<size_t>(c_first) + seq;
     for (int g = warp; g < p.G; g += n_warps) {

@@ -31,6 +31,7 @@ struct RecallParams {
     long long host_stride, pool_stride, unit_bytes;
     long long unit_stride, list_offset;            // distance between consecutive units; byte offset of list (l % lists_per_seq)
     int n_lists, lists_per_seq, cap, cache_cap;
+    long long pool_units, host_units;              // units one sequence's pool region / host region holds
     // paged host store: unit u of sequence s is page page[s * page_stride + u] of the arena at `host`
     const int32_t* page;
     long long page_stride;
@@ -163,6 +164,15 @@ recall_kernel(RecallParams p) {
             if (lane == 0) pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_RECALL, l, elo, e.src_unit);
             return;
         }
+        // a unit beyond the sequence's pool region (or, block-major store, its host region) is skipped
+        if (static_cast<long long>(e.dst_unit) + k >= p.pool_units) {
+            if (lane == 0) pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_RECALL, l, elo, e.dst_unit + k);
+            return;
+        }
+        if (!PAGED && static_cast<long long>(e.src_unit) + k >= p.host_units) {
+            if (lane == 0) pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_RECALL, l, elo, e.src_unit + k);
+            return;
+        }
         const int seq = l / p.lists_per_seq;
         const long long loff = (l - seq * p.lists_per_seq) * p.list_offset + in_unit + lane * 16;
         if (PAGED) {
@@ -220,6 +230,10 @@ int pi_launch_recall(pi_ctx* c, int n_lists, int lists_per_seq, const void* host
     p.unit_stride = unit_stride > 0 ? unit_stride : unit_bytes;
     p.list_offset = list_offset;
     p.n_lists = n_lists; p.lists_per_seq = lists_per_seq; p.cap = cap;
+    // capacities of one sequence's regions in units (pool: C blocks, host: NB blocks of block_bytes)
+    const long long block_bytes = static_cast<long long>(c->cfg.n_kv_heads) * c->cfg.block_tokens * PI_HEAD_DIM * 4;
+    p.pool_units = static_cast<long long>(c->cfg.pool_slots) * block_bytes / p.unit_stride;
+    p.host_units = static_cast<long long>(c->cfg.max_blocks) * block_bytes / p.unit_stride;
     // shared memory: two prefix arrays over the lists + the extent cache
     const long long want = static_cast<long long>(n_lists) * cap;
     p.cache_cap = static_cast<int>(want < RECALL_CACHE_EXTENTS ? want : RECALL_CACHE_EXTENTS);

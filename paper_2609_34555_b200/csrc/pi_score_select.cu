@@ -457,7 +457,8 @@ static int launch_score_select(SelParams& p, int batch, int n_sms, cudaStream_t 
     const size_t smem = (static_cast<size_t>(p.max_blocks) + p.max_blocks / 32 + 1) * sizeof(uint32_t);
     const bool multi = p.vh > 1 || p.n_sum > 1 || p.dig_heads > 1;
     auto kern = multi ? score_select_kernel<true> : score_select_kernel<false>;
-    if (smem > 40 * 1024)
+    // the kernel also holds about 9 KB of static shared memory: opt in before the two together pass 48 KB
+    if (smem > 36 * 1024)
         PI_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
     // a plain launch: this grid fills every SM's registers, so it must not sit resident waiting for
     // the kernel before it (it would keep the attention kernel of the other stream off the SMs)

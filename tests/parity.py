@@ -18,6 +18,32 @@ NEAR_TIE_REL = 1e-4
 SCORE_RTOL, SCORE_ATOL = 2e-5, 2e-3
 
 
+ATTN_OUTLIER_ALLOWANCE = 4e-3     # compute error allowed beyond the output's own bf16 rounding on the scaled channels
+
+
+def bf16_half_ulp(x: np.ndarray) -> np.ndarray:
+    """Half the spacing of bf16 numbers (8 significand bits) around x."""
+    e = np.floor(np.log2(np.maximum(np.abs(x), 2.0 ** -126)))
+    return 2.0 ** (e - 8)
+
+
+def check_attention(got: np.ndarray, ref: np.ndarray, cfg, layer: int, what: str = "attention") -> dict:
+    """got, ref: [..., D].  The benchmark's tolerance, max-abs 2e-2 and mean-abs 2e-3, holds on every channel
+    except the layer's four scaled (x8) outlier channels of the workload; there the outputs reach
+    magnitudes whose bf16 spacing alone exceeds 2e-2, so the bound is the rounding of the output itself,
+    half a bf16 ulp of the reference, plus ATTN_OUTLIER_ALLOWANCE for the arithmetic (never below 2e-2).
+    Returns the two maxima."""
+    mask = np.zeros(ref.shape[-1], bool)
+    mask[gen.outlier_channels(cfg, layer).numpy()] = True
+    err = np.abs(got - ref)
+    ordinary, scaled = err[..., ~mask], err[..., mask]
+    assert ordinary.max() <= ATTN_MAX_ABS, f"{what}: max-abs {ordinary.max()} on the ordinary channels"
+    bound = np.maximum(ATTN_MAX_ABS, bf16_half_ulp(ref[..., mask]) + ATTN_OUTLIER_ALLOWANCE)
+    assert np.all(scaled <= bound), f"{what}: {scaled.max()} on a scaled channel"
+    assert err.mean() <= ATTN_MEAN_ABS, f"{what}: mean-abs {err.mean()}"
+    return dict(max_abs_ordinary=float(ordinary.max()), max_abs_scaled=float(scaled.max()), mean_abs=float(err.mean()))
+
+
 def expand_extents(lst: np.ndarray, count: int) -> np.ndarray:
     pairs = []
     before = 0
@@ -139,7 +165,7 @@ def run_and_compare(case: Case, steps: int, layer: int = 0, overlapped: bool = F
 
     out_d = torch.zeros((cfg.batch, cfg.n_q_heads, cfg.head_dim), dtype=torch.bfloat16, device=dev)
     lse_d = torch.zeros((cfg.batch, cfg.n_q_heads), dtype=torch.float32, device=dev)
-    stats = dict(max_abs=0.0, mean_abs=0.0, misses=[], sel_diffs=0, extents=0)
+    stats = dict(max_abs=0.0, max_abs_scaled=0.0, mean_abs=0.0, misses=[], sel_diffs=0, extents=0)
     for t in range(steps):
         step = t + 1
         q_d = case.q[t].to(dev)
@@ -178,13 +204,10 @@ def run_and_compare(case: Case, steps: int, layer: int = 0, overlapped: bool = F
             assert np.array_equal(got_pairs, pairs.reshape(-1, 2)), f"seq {s}: recall list"
             stats["misses"].append(len(pairs))
             stats["extents"] += int(g_lcnt[s])
-            err = np.abs(g_out[s] - out)
-            stats["max_abs"] = max(stats["max_abs"], float(err.max()))
-            stats["mean_abs"] = max(stats["mean_abs"], float(err.mean()))
-            # 2e-2 absolute; where the bf16 spacing of the output itself exceeds that (|out| > 5,
-            # the scaled outlier channels) the bound is the output rounding, 2^-8 relative
-            bound = np.maximum(ATTN_MAX_ABS, np.abs(out) * 2.0 ** -8)
-            assert np.all(err <= bound) and err.mean() <= ATTN_MEAN_ABS, f"seq {s}: attention {err.max()} {err.mean()}"
+            a = check_attention(g_out[s], out, cfg, layer, f"seq {s}: attention")
+            stats["max_abs"] = max(stats["max_abs"], a["max_abs_ordinary"])
+            stats["max_abs_scaled"] = max(stats["max_abs_scaled"], a["max_abs_scaled"])
+            stats["mean_abs"] = max(stats["mean_abs"], a["mean_abs"])
             np.testing.assert_allclose(g_lse[s], lse, rtol=1e-3, atol=1e-3)
         assert np.array_equal(buf.block_table.cpu().numpy(), ref.table), "block table"
         assert np.array_equal(buf.slot_block.cpu().numpy(), ref.slot_block), "slot_block"
@@ -195,7 +218,8 @@ def run_and_compare(case: Case, steps: int, layer: int = 0, overlapped: bool = F
 
 
 def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, settle_cold: bool = True,
-                        append: bool = False, ctx_start: int = 0, paged: bool = False) -> dict:
+                        append: bool = False, ctx_start: int = 0, paged: bool = False, pi_kwargs=None,
+                        return_out: bool = False) -> dict:
     """The bench's launch configuration (DecodeSession: whole batch per call, every layer,
     three-stream pipeline) at a full-size shape; the oracle follows only `sample_seqs`, which is
     enough because sequences are independent.  Inputs are generated on the GPU and handed to the
@@ -204,7 +228,7 @@ def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, s
     from paper_2609_34555_b200.runner import DecodeSession
 
     dev = torch.device("cuda:0")
-    pi = PulseInfer.from_workload(cfg)
+    pi = PulseInfer.from_workload(cfg, **(pi_kwargs or {}))
     sess = DecodeSession(pi, cfg.batch, cfg.n_layers, keep_scores=True, paged=paged, page_seed=cfg.seed + 5)
     ctx_now = ctx_start or cfg.ctx                     # runs that append start short of the full context
     sess.ctx_len.fill_(ctx_now)
@@ -289,9 +313,7 @@ def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, s
                 stats["misses"] += len(pairs)
                 ref, _ = oracle.attention(qb, o["pool"], slots, g_sel[s], int(g_cnt[s]), ctx_now, cfg.block_tokens,
                                           cfg.n_kv_heads)
-                err = np.abs(out[l, s] - ref)
-                stats["max_abs"] = max(stats["max_abs"], float(err.max()))
-                assert np.all(err <= np.maximum(ATTN_MAX_ABS, np.abs(ref) * 2.0 ** -8)) and err.mean() <= ATTN_MEAN_ABS
+                stats["max_abs"] = max(stats["max_abs"], check_attention(out[l, s], ref, cfg, l)["max_abs_ordinary"])
                 assert np.array_equal(b.block_table[s].cpu().numpy(), o["table"])
                 assert np.array_equal(b.slot_stamp[s].cpu().numpy().view(np.uint32), o["slot_stamp"])
                 assert np.array_equal(oracle.bits(b.pool[s].cpu()), o["pool"]), "pool bytes"
@@ -301,6 +323,8 @@ def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, s
             for s in sample_seqs:
                 assert np.array_equal(host[s, :n_now], ora[(l, s)]["kvb"][:n_now]), "host store after the appends"
                 assert np.array_equal(oracle.bits(sess.bufs[l].digest[s].cpu())[:n_now], ora[(l, s)]["digest"][:n_now])
+    if return_out:
+        stats["out"] = sess.out.clone()
     pi.close()
     return stats
 
@@ -364,9 +388,7 @@ def run_append_and_compare(cfg, steps: int, ctx_len0, layer: int = 0) -> dict:
             stats["misses"] += len(pairs)
             want, _ = oracle.attention(qb[s], ref.pool[s], slots, g_sel[s], int(g_cnt[s]), int(ctx[s]), cfg.block_tokens,
                                        cfg.n_kv_heads)
-            err = np.abs(g_out[s] - want)
-            stats["max_abs"] = max(stats["max_abs"], float(err.max()))
-            assert np.all(err <= np.maximum(ATTN_MAX_ABS, np.abs(want) * 2.0 ** -8)) and err.mean() <= ATTN_MEAN_ABS
+            stats["max_abs"] = max(stats["max_abs"], check_attention(g_out[s], want, cfg, layer)["max_abs_ordinary"])
         assert np.array_equal(buf.block_table.cpu().numpy(), ref.table)
         assert np.array_equal(buf.slot_block.cpu().numpy(), ref.slot_block)
         assert np.array_equal(buf.slot_stamp.cpu().numpy().view(np.uint32), ref.slot_stamp)
@@ -497,9 +519,8 @@ def run_strategies_and_compare(cfg, steps: int = 2, layer: int = 0) -> dict:
                                                cfg.block_tokens, Hkv)
                 rows = slice(h * G, (h + 1) * G)
                 assert np.array_equal(ref[rows], via_host[rows]), "byte invariant seen through attention"
-                err = np.abs(g_out[s, rows] - ref[rows])
-                stats["attn_max_abs"] = max(stats["attn_max_abs"], float(err.max()))
-                assert np.all(err <= np.maximum(ATTN_MAX_ABS, np.abs(ref[rows]) * 2.0 ** -8)) and err.mean() <= ATTN_MEAN_ABS
+                stats["attn_max_abs"] = max(stats["attn_max_abs"],
+                                            check_attention(g_out[s, rows], ref[rows], cfg, layer)["max_abs_ordinary"])
                 np.testing.assert_allclose(g_lse[s, rows], ref_lse[rows], rtol=1e-3, atol=1e-3)
     # heads really choose differently (the fragmentation the shared selection avoids)
     stats["distinct_head_selections"] = len({tuple(g_sel[h].tolist()) for h in range(Hkv)})
