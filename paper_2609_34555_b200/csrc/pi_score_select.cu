@@ -16,12 +16,18 @@
 // *varying* bits narrows [lo, hi] until the k-th key is isolated, then one ordered
 // compaction emits the result in ascending block order.
 #include "pi_common.cuh"
+#include "pi_score_core.cuh"
 
 namespace {
 
+using pi_score::BLOCKS_PER_WARP;
+using pi_score::dot8;
+using pi_score::float_key;
+using pi_score::ld_stream16;
+using pi_score::padded;
+
 constexpr int SCORE_THREADS = 512;
 constexpr int SCORE_WARPS = SCORE_THREADS / 32;
-constexpr int BLOCKS_PER_WARP = 8;               // 8 independent 16-byte loads per lane
 constexpr int SCORE_CHUNK = SCORE_WARPS * BLOCKS_PER_WARP;   // 128 blocks (64 KB of digests) per CTA
 constexpr int BINS = PI_SELECT_BINS;
 constexpr int BINS_PER_THREAD = BINS / SCORE_THREADS;
@@ -45,35 +51,6 @@ struct SelParams {
     //   headwise:            vh Hkv, n_sum 1, h_base 0, hv_step 1, dig_heads Hkv
     int vh, n_sum, h_base, hv_step, dig_heads;
 };
-
-// Shared arrays that one thread walks with a stride of several words are stored with one
-// pad word every 32 entries, which keeps both the strided and the unit-stride walks free
-// of bank conflicts.
-__device__ __forceinline__ int padded(int i) { return i + (i >> 5); }
-
-__device__ __forceinline__ uint32_t float_key(float s) {
-    uint32_t u = __float_as_uint(s + 0.0f);       // -0 -> +0
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
-__device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
-}
-
-__device__ __forceinline__ float dot8(uint4 v, const float (&w)[8]) {
-    float2 a = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&v.x));
-    float2 b = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&v.y));
-    float2 c = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&v.z));
-    float2 d = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&v.w));
-    float s0 = a.x * w[0] + b.x * w[2];
-    float s1 = a.y * w[1] + b.y * w[3];
-    s0 = fmaf(c.x, w[4], s0); s1 = fmaf(c.y, w[5], s1);
-    s0 = fmaf(d.x, w[6], s0); s1 = fmaf(d.y, w[7], s1);
-    return s0 + s1;
-}
 
 // Block-wide exclusive scan (SCORE_THREADS threads, all must call).
 __device__ __forceinline__ unsigned block_excl_scan(unsigned v, unsigned* warp_tot, unsigned& total) {
@@ -302,31 +279,8 @@ score_select_kernel(SelParams p) {
                 if (b0 + i < p.max_blocks) v[i] = ld_stream16(dg + static_cast<size_t>(b0 + i) * dig_heads * 32 + lane);
             }
             if (c == f || n_sum > 1) {
-                // lanes 0-15 hold Q- for channels 8*lane.., lanes 16-31 hold Q+ for channels 8*(lane-16)..
-#pragma unroll
-                for (int i = 0; i < 8; ++i) w[i] = 0.f;
-                const int d0 = (lane & 15) * 8;
-                const bool plus = lane >= 16;
-                const __nv_bfloat16* qh = p.q + (static_cast<size_t>(rseq) * p.Hq + static_cast<size_t>(head) * p.G) * PI_HEAD_DIM + d0;
-                // the group's query rows are fetched four at a time so their latencies overlap
-                for (int g0 = 0; g0 < p.G; g0 += 4) {
-                    uint4 qv[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        qv[j] = make_uint4(0, 0, 0, 0);
-                        if (g0 + j < p.G) qv[j] = *reinterpret_cast<const uint4*>(qh + static_cast<size_t>(g0 + j) * PI_HEAD_DIM);
-                    }
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&qv[j]);
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            float2 fv = __bfloat1622float2(h2[i]);
-                            w[2 * i] += plus ? fmaxf(fv.x, 0.f) : fminf(fv.x, 0.f);
-                            w[2 * i + 1] += plus ? fmaxf(fv.y, 0.f) : fminf(fv.y, 0.f);
-                        }
-                    }
-                }
+                pi_score::load_q_weights(p.q + (static_cast<size_t>(rseq) * p.Hq + static_cast<size_t>(head) * p.G) * PI_HEAD_DIM,
+                                         p.G, lane, w);
             }
             if (c == f && hh == 0) {
                 int ctx = p.ctx_len[rseq];
@@ -344,29 +298,7 @@ score_select_kernel(SelParams p) {
 #pragma unroll
             for (int i = 0; i < BLOCKS_PER_WARP; ++i) s[i] = acc[i];
 
-            // transposed warp reduction: 8 values x 32 lanes -> lane group (lane>>2) owns block (lane>>2)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const bool up = lane & 16;
-                float send = up ? s[i] : s[i + 4];
-                float keep = up ? s[i + 4] : s[i];
-                s[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
-            }
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                const bool up = lane & 8;
-                float send = up ? s[i] : s[i + 2];
-                float keep = up ? s[i + 2] : s[i];
-                s[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
-            }
-            {
-                const bool up = lane & 4;
-                float send = up ? s[0] : s[1];
-                float keep = up ? s[1] : s[0];
-                s[0] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-            }
-            s[0] += __shfl_xor_sync(0xffffffffu, s[0], 2);
-            s[0] += __shfl_xor_sync(0xffffffffu, s[0], 1);
+            pi_score::reduce8(s, lane);
             const int b = b0 + (lane >> 2);
             if ((lane & 3) == 0 && b < n_blocks) p.scores[static_cast<size_t>(seq) * p.max_blocks + b] = s[0];
         }

@@ -223,7 +223,8 @@ def test_sequences_that_no_cta_splits_pipelined_and_repeatable():
     case; several pipelined steps; two runs give the same bits."""
     from tests.parity import make_case, run_and_compare
     from tests.parity import run_session_sampled
-    one_block = tiny_config(batch=4, ctx=16, n_q_heads=8, n_kv_heads=2, budget_blocks=4, resident_frac=1.0)
+    one_block = tiny_config(batch=4, ctx=16, n_q_heads=8, n_kv_heads=2, budget_blocks=2, resident_frac=1.0,
+                            sink_tokens=0, local_tokens=16)
     for ctas in (1, 2, 4):
         run_and_compare(make_case(one_block, steps=2), steps=2, overlapped=True, pi_kwargs=dict(attn_ctas=ctas))
     cfg = tiny_config(batch=6, ctx=2000, n_q_heads=16, n_kv_heads=4, budget_blocks=24, resident_frac=0.4, n_layers=3)
