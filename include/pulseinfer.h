@@ -156,7 +156,24 @@ int pi_diff_misses(pi_ctx* ctx, int layer, int batch, uint32_t step, const int32
                    int32_t* sel_slots_dev, pi_extent* recall_list_dev, int32_t* recall_count_dev,
                    void* stream);
 
-/* The same with the step number read from device memory when the kernel runs (one uint32, > 0), so
+/* Steps 1 and 2 of the workflow (Sec. 2.2: sparse selection, then B_recall = B_topk \ B_gpu) in ONE launch:
+ * pi_score_select followed by pi_diff_misses with the same arguments and the same results, bit for bit
+ * (selection, slots, tables, stamps, recall list).  The CTA that selects for a sequence diffs its selection
+ * while it is still in shared memory, and what the diff needs besides the selection is fetched while the
+ * digests stream in, so the launch and the global round trips between the two steps disappear.
+ * Arguments as in the two calls; scores_dev may be NULL.  The _devstep form reads the step number
+ * from device memory like pi_diff_misses_devstep. */
+int pi_score_select_diff(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* q_dev, const void* digest_dev,
+                         const int32_t* ctx_len_dev, int32_t* sel_blocks_dev, int32_t* sel_count_dev, float* scores_dev,
+                         int32_t* block_table_dev, int32_t* slot_block_dev, uint32_t* slot_stamp_dev,
+                         int32_t* sel_slots_dev, pi_extent* recall_list_dev, int32_t* recall_count_dev, void* stream);
+int pi_score_select_diff_devstep(pi_ctx* ctx, int layer, int batch, const uint32_t* step_dev, const void* q_dev,
+                                 const void* digest_dev, const int32_t* ctx_len_dev, int32_t* sel_blocks_dev,
+                                 int32_t* sel_count_dev, float* scores_dev, int32_t* block_table_dev,
+                                 int32_t* slot_block_dev, uint32_t* slot_stamp_dev, int32_t* sel_slots_dev,
+                                 pi_extent* recall_list_dev, int32_t* recall_count_dev, void* stream);
+
+/* pi_diff_misses with the step number read from device memory when the kernel runs (one uint32, > 0), so
  * that a CUDA graph holding the call can be replayed for later steps: the caller advances *step_dev
  * between replays (in the graph or outside).  The paper has no counterpart. */
 int pi_diff_misses_devstep(pi_ctx* ctx, int layer, int batch, const uint32_t* step_dev,

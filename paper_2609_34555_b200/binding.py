@@ -22,7 +22,7 @@ ERR_NAMES = {
 }
 EXTENT_DTYPE = torch.int32      # a pi_extent is four int32: src_unit, dst_unit, n_units, units_before
 
-EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_score_select_noalloc", "pi_score_select_strategy", "pi_diff_misses", "pi_diff_misses_devstep", "pi_recall_gather_scatter",
+EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_score_select_diff", "pi_score_select_diff_devstep", "pi_score_select_noalloc", "pi_score_select_strategy", "pi_diff_misses", "pi_diff_misses_devstep", "pi_recall_gather_scatter",
            "pi_recall_gather_scatter_paged", "pi_sparse_decode_attn", "pi_sparse_decode_attn_headwise", "pi_append_kv", "pi_append_kv_paged", "pi_append_kv_devstep", "pi_build_digests", "pi_build_digests_all", "pi_table_init", "pi_h2d_copy_ms",
            "pi_get_status", "pi_get_stats", "pi_clear_status", "pi_strerror"]
 
@@ -57,6 +57,8 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.pi_destroy.argtypes = [c_void_p]
     lib.pi_score_select.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, vp, vp]
     lib.pi_score_select_noalloc.argtypes = [c_int] * 9 + [vp, vp, i32p, i32p, i32p, i32p, vp]
+    lib.pi_score_select_diff.argtypes = [c_void_p, c_int, c_int, c_uint32, vp, vp, i32p, i32p, i32p, vp, i32p, i32p, u32p, i32p, vp, i32p, vp]
+    lib.pi_score_select_diff_devstep.argtypes = [c_void_p, c_int, c_int, u32p, vp, vp, i32p, i32p, i32p, vp, i32p, i32p, u32p, i32p, vp, i32p, vp]
     lib.pi_diff_misses.argtypes = [c_void_p, c_int, c_int, c_uint32, i32p, i32p, i32p, i32p, i32p, u32p, i32p, vp, i32p, vp]
     lib.pi_diff_misses_devstep.argtypes = [c_void_p, c_int, c_int, u32p, i32p, i32p, i32p, i32p, i32p, u32p, i32p, vp, i32p, vp]
     lib.pi_recall_gather_scatter.argtypes = [c_void_p, c_int, c_int, c_int, vp, c_int64, vp, c_int64, vp, c_int32, i32p,
@@ -180,6 +182,23 @@ class PulseInfer:
             _dev(ctx_len, torch.int32, "ctx_len"), _dev(sel_blocks, torch.int32, "sel_blocks"),
             _dev(sel_count, torch.int32, "sel_count"),
             None if scores is None else _dev(scores, torch.float32, "scores"), _stream(stream)))
+
+    def score_select_diff(self, layer: int, step, q, digest, ctx_len, sel_blocks, sel_count, block_table, slot_block,
+                          slot_stamp, sel_slots, recall_list, recall_count, scores=None, stream=None) -> None:
+        """score_select and diff_misses in one launch (same results).  step: a positive int, or a
+        one-element int32 CUDA tensor read when the kernel runs (calls captured into a CUDA graph)."""
+        batch = q.shape[0]
+        dev_step = isinstance(step, torch.Tensor)
+        fn = self._lib.pi_score_select_diff_devstep if dev_step else self._lib.pi_score_select_diff
+        _check("pi_score_select_diff_devstep" if dev_step else "pi_score_select_diff", fn(
+            self._ctx, layer, batch, _dev(step, torch.int32, "step") if dev_step else step,
+            _dev(q, torch.bfloat16, "q"), _dev(digest, torch.bfloat16, "digest"), _dev(ctx_len, torch.int32, "ctx_len"),
+            _dev(sel_blocks, torch.int32, "sel_blocks"), _dev(sel_count, torch.int32, "sel_count"),
+            None if scores is None else _dev(scores, torch.float32, "scores"),
+            _dev(block_table, torch.int32, "block_table"), _dev(slot_block, torch.int32, "slot_block"),
+            _dev(slot_stamp, torch.int32, "slot_stamp"), _dev(sel_slots, torch.int32, "sel_slots"),
+            _dev(recall_list, EXTENT_DTYPE, "recall_list"), _dev(recall_count, torch.int32, "recall_count"),
+            _stream(stream)))
 
     AVERAGE, HEADWISE = 1, 2
 

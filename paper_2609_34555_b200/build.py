@@ -14,7 +14,7 @@ CSRC = PKG / "csrc"
 INCLUDE = PKG.parent / "include"
 LIB = PKG / "libpulseinfer_b200.so"
 
-SOURCES = ["pi_api.cu", "pi_score_select.cu", "pi_diff_misses.cu", "pi_recall.cu", "pi_attn.cu",
+SOURCES = ["pi_api.cu", "pi_score_select.cu", "pi_select_diff.cu", "pi_diff_misses.cu", "pi_recall.cu", "pi_attn.cu",
            "pi_helpers.cu", "pi_append.cu"]
 
 
@@ -38,6 +38,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-Xcompiler", "-fPIC", "-shared", f"-I{INCLUDE}", f"-I{CSRC}",
            "-o", str(tmp)] + [str(s) for s in sources()]
+    cmd[1:1] = os.environ.get("PI_NVCC_FLAGS", "").split()       # extra flags for experiments (-D..., -Xptxas=-v)
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     subprocess.check_call(cmd)

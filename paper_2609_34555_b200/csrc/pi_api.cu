@@ -47,6 +47,8 @@ extern "C" int pi_create(const pi_config* cfg, pi_ctx** out) {
     if (!c) return PI_ERR_INVALID_ARG;
     std::memset(c, 0, sizeof(*c));
     c->cfg = *cfg;
+    for (int i = 0; i < 2; ++i)
+        for (int j = 0; j < 4; ++j) c->sd_resident_clusters[i][j] = -1;
     c->solo_head = static_cast<int32_t*>(std::malloc(sizeof(int32_t) * cfg->n_layers));
     std::memcpy(c->solo_head, cfg->solo_head, sizeof(int32_t) * cfg->n_layers);
     c->cfg.solo_head = c->solo_head;
@@ -120,9 +122,48 @@ extern "C" int pi_score_select(pi_ctx* ctx, int layer, int batch, const void* q_
     if (rc != PI_OK) return rc;
     if (!q_dev || !digest_dev || !ctx_len_dev || !sel_blocks_dev || !sel_count_dev) return PI_ERR_INVALID_ARG;
     if (!pi_aligned16(q_dev) || !pi_aligned16(digest_dev)) return PI_ERR_BAD_ALIGN;
-    return pi_launch_score_select(ctx, ctx->solo_head[layer], batch, q_dev, digest_dev, ctx_len_dev,
-                                  sel_blocks_dev, sel_count_dev, scores_dev ? scores_dev : ctx->scores,
-                                  ctx->sel_counters, static_cast<cudaStream_t>(stream));
+    return pi_launch_select_cluster(ctx, ctx->solo_head[layer], batch, q_dev, digest_dev, ctx_len_dev, sel_blocks_dev,
+                                    sel_count_dev, scores_dev, 0, 0, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
+                                    nullptr, static_cast<cudaStream_t>(stream));
+}
+
+static int select_diff_call(pi_ctx* ctx, int layer, int batch, uint32_t step, const uint32_t* step_dev, const void* q_dev,
+                            const void* digest_dev, const int32_t* ctx_len_dev, int32_t* sel_blocks_dev,
+                            int32_t* sel_count_dev, float* scores_dev, int32_t* block_table_dev, int32_t* slot_block_dev,
+                            uint32_t* slot_stamp_dev, int32_t* sel_slots_dev, pi_extent* recall_list_dev,
+                            int32_t* recall_count_dev, void* stream) {
+    int rc = check_call(ctx, layer, batch);
+    if (rc != PI_OK) return rc;
+    if (!q_dev || !digest_dev || !ctx_len_dev || !sel_blocks_dev || !sel_count_dev || !block_table_dev ||
+        !slot_block_dev || !slot_stamp_dev || !sel_slots_dev || !recall_list_dev || !recall_count_dev ||
+        (!step_dev && step == 0))
+        return PI_ERR_INVALID_ARG;
+    if (!pi_aligned16(q_dev) || !pi_aligned16(digest_dev) || !pi_aligned16(recall_list_dev)) return PI_ERR_BAD_ALIGN;
+    return pi_launch_select_cluster(ctx, ctx->solo_head[layer], batch, q_dev, digest_dev, ctx_len_dev, sel_blocks_dev,
+                                    sel_count_dev, scores_dev, 1, step, step_dev, block_table_dev, slot_block_dev,
+                                    slot_stamp_dev, sel_slots_dev, recall_list_dev, recall_count_dev,
+                                    static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int pi_score_select_diff(pi_ctx* ctx, int layer, int batch, uint32_t step, const void* q_dev,
+                                    const void* digest_dev, const int32_t* ctx_len_dev, int32_t* sel_blocks_dev,
+                                    int32_t* sel_count_dev, float* scores_dev, int32_t* block_table_dev,
+                                    int32_t* slot_block_dev, uint32_t* slot_stamp_dev, int32_t* sel_slots_dev,
+                                    pi_extent* recall_list_dev, int32_t* recall_count_dev, void* stream) {
+    return select_diff_call(ctx, layer, batch, step, nullptr, q_dev, digest_dev, ctx_len_dev, sel_blocks_dev, sel_count_dev,
+                            scores_dev, block_table_dev, slot_block_dev, slot_stamp_dev, sel_slots_dev, recall_list_dev,
+                            recall_count_dev, stream);
+}
+
+extern "C" int pi_score_select_diff_devstep(pi_ctx* ctx, int layer, int batch, const uint32_t* step_dev, const void* q_dev,
+                                            const void* digest_dev, const int32_t* ctx_len_dev, int32_t* sel_blocks_dev,
+                                            int32_t* sel_count_dev, float* scores_dev, int32_t* block_table_dev,
+                                            int32_t* slot_block_dev, uint32_t* slot_stamp_dev, int32_t* sel_slots_dev,
+                                            pi_extent* recall_list_dev, int32_t* recall_count_dev, void* stream) {
+    if (!step_dev) return PI_ERR_INVALID_ARG;
+    return select_diff_call(ctx, layer, batch, 0, step_dev, q_dev, digest_dev, ctx_len_dev, sel_blocks_dev, sel_count_dev,
+                            scores_dev, block_table_dev, slot_block_dev, slot_stamp_dev, sel_slots_dev, recall_list_dev,
+                            recall_count_dev, stream);
 }
 
 extern "C" int pi_score_select_strategy(pi_ctx* ctx, int strategy, int layer, int batch, const void* q_dev,

@@ -69,6 +69,8 @@ struct pi_ctx {
     long long pool_map_slots;
     int pool_map_headwise;       // box of the cached map: all KV heads of a block (0) or one head (1)
     void* encode_tiled_fn;
+    // clusters of 2^i CTAs of the selection kernel that are resident at once, [plain | fused][i]; -1 = not asked yet
+    int sd_resident_clusters[2][4];
 };
 
 struct pi_status_ref {
@@ -106,6 +108,11 @@ __device__ __forceinline__ int pi_ceil_div(int a, int b) { return (a + b - 1) / 
 int pi_launch_score_select(pi_ctx*, int h_star, int batch, const void* q, const void* digest,
                            const int32_t* ctx_len, int32_t* sel, int32_t* sel_count, float* scores,
                            unsigned int* counters, cudaStream_t);
+// fused != 0: the diff of the selection runs in the same launch (the diff arguments are then required)
+int pi_launch_select_cluster(pi_ctx*, int h_star, int batch, const void* q, const void* digest, const int32_t* ctx_len,
+                             int32_t* sel, int32_t* sel_count, float* scores, int fused, uint32_t step,
+                             const uint32_t* step_dev, int32_t* table, int32_t* slot_block, uint32_t* slot_stamp,
+                             int32_t* sel_slots, pi_extent* list, int32_t* count, cudaStream_t);
 int pi_launch_score_select_strategy(pi_ctx*, int strategy, int batch, const void* q, const void* digest_all,
                                     const int32_t* ctx_len, int32_t* sel, int32_t* sel_count, float* scores,
                                     unsigned int* counters, cudaStream_t);

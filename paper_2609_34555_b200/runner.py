@@ -65,11 +65,17 @@ class RecallPath:
         pi.recall_gather_scatter(layer, host_kv, buf.pool, fill.contiguous(), n.contiguous(), page_table=page_table)
 
     def select_and_recall(self, layer: int, step: int, buf: LayerBuffers, q: torch.Tensor, ctx_len: torch.Tensor,
-                          host_kv: torch.Tensor, stream=None) -> None:
+                          host_kv: torch.Tensor, stream=None, fused: bool = True) -> None:
+        """fused: selection and diff in one launch (pi_score_select_diff); else the two calls."""
         pi = self.pi
-        pi.score_select(layer, q, buf.digest, ctx_len, buf.sel_blocks, buf.sel_count, buf.scores, stream=stream)
-        pi.diff_misses(layer, step, ctx_len, buf.sel_blocks, buf.sel_count, buf.block_table, buf.slot_block,
-                       buf.slot_stamp, buf.sel_slots, buf.recall_list, buf.recall_count, stream=stream)
+        if fused:
+            pi.score_select_diff(layer, step, q, buf.digest, ctx_len, buf.sel_blocks, buf.sel_count, buf.block_table,
+                                 buf.slot_block, buf.slot_stamp, buf.sel_slots, buf.recall_list, buf.recall_count,
+                                 scores=buf.scores, stream=stream)
+        else:
+            pi.score_select(layer, q, buf.digest, ctx_len, buf.sel_blocks, buf.sel_count, buf.scores, stream=stream)
+            pi.diff_misses(layer, step, ctx_len, buf.sel_blocks, buf.sel_count, buf.block_table, buf.slot_block,
+                           buf.slot_stamp, buf.sel_slots, buf.recall_list, buf.recall_count, stream=stream)
         pi.recall_gather_scatter(layer, host_kv, buf.pool, buf.recall_list, buf.recall_count, stream=stream)
 
     def attention(self, layer: int, buf: LayerBuffers, q: torch.Tensor, ctx_len: torch.Tensor, out: torch.Tensor,
@@ -78,19 +84,21 @@ class RecallPath:
                                    lse, stream=stream)
 
     def layer_step(self, layer: int, step: int, buf: LayerBuffers, q: torch.Tensor, ctx_len: torch.Tensor,
-                   host_kv: torch.Tensor, out: torch.Tensor, lse: Optional[torch.Tensor] = None) -> None:
-        """Serial form: all four calls on the current stream."""
-        self.select_and_recall(layer, step, buf, q, ctx_len, host_kv)
+                   host_kv: torch.Tensor, out: torch.Tensor, lse: Optional[torch.Tensor] = None,
+                   fused: bool = True) -> None:
+        """Serial form: all calls on the current stream."""
+        self.select_and_recall(layer, step, buf, q, ctx_len, host_kv, fused=fused)
         self.attention(layer, buf, q, ctx_len, out, lse)
 
     def layer_step_overlapped(self, layer: int, step: int, buf: LayerBuffers, q: torch.Tensor, ctx_len: torch.Tensor,
-                              host_kv: torch.Tensor, out: torch.Tensor, lse: Optional[torch.Tensor] = None) -> None:
+                              host_kv: torch.Tensor, out: torch.Tensor, lse: Optional[torch.Tensor] = None,
+                              fused: bool = True) -> None:
         """Selection, diff and recall run on the side stream; attention waits for the
         recall event on the current stream, so the recall of the next call can overlap it."""
         main = torch.cuda.current_stream()
         self._ev_in.record(main)
         self.side.wait_event(self._ev_in)
-        self.select_and_recall(layer, step, buf, q, ctx_len, host_kv, stream=self.side)
+        self.select_and_recall(layer, step, buf, q, ctx_len, host_kv, stream=self.side, fused=fused)
         ev = torch.cuda.Event()
         ev.record(self.side)
         main.wait_event(ev)
@@ -106,7 +114,7 @@ class StageTimer:
     afterwards (`light_summary`).  Extra events between the kernels of the recall streams cost
     the pipelined step about 6 % of its rate, which is why the timed region uses this form."""
 
-    STAGES = ("append", "score_select", "diff", "recall", "attn")
+    STAGES = ("append", "select_diff", "score_select", "diff", "recall", "attn")
 
     def __init__(self, stages=None, light: bool = False):
         self.stages = tuple(stages) if stages else self.STAGES
@@ -208,8 +216,9 @@ class DecodeSession:
 
     def __init__(self, pi: PulseInfer, batch: int, n_layers: int, host_layers: Optional[int] = None,
                  device="cuda", keep_scores: bool = False, paged: bool = False, page_seed: int = 0,
-                 recall_streams: int = 2):
+                 recall_streams: int = 2, fused_select_diff: bool = True):
         c = pi.cfg
+        self.fused_select_diff = fused_select_diff     # selection + diff in one launch (pi_score_select_diff)
         self.pi, self.batch, self.n_layers = pi, batch, n_layers
         self.host_layers = n_layers if host_layers is None else max(1, min(host_layers, n_layers))
         self.device = torch.device(device)
@@ -330,12 +339,21 @@ class DecodeSession:
                              b.slot_block, b.slot_stamp, b.digest, page_table=pt, stream=sel_s)
                 if ta is not None:
                     tm.add("append", ta, tm.mark(sel_s))
-            t0 = tm.mark(sel_s) if tm and tm.wants("score_select") else None
-            pi.score_select(l, q[l], b.digest, self.ctx_len, b.sel_blocks, b.sel_count, b.scores, stream=sel_s)
-            t1 = tm.mark(sel_s) if tm and (tm.wants("score_select") or tm.wants("diff")) else None
-            pi.diff_misses(l, step, self.ctx_len, b.sel_blocks, b.sel_count, b.block_table, b.slot_block,
-                           b.slot_stamp, b.sel_slots, b.recall_list, b.recall_count, stream=sel_s)
-            t2 = tm.mark(sel_s) if tm and tm.wants("diff") else None
+            if self.fused_select_diff:
+                t0 = tm.mark(sel_s) if tm and tm.wants("select_diff") else None
+                pi.score_select_diff(l, step, q[l], b.digest, self.ctx_len, b.sel_blocks, b.sel_count, b.block_table,
+                                     b.slot_block, b.slot_stamp, b.sel_slots, b.recall_list, b.recall_count,
+                                     scores=b.scores, stream=sel_s)
+                if t0 is not None:
+                    tm.add("select_diff", t0, tm.mark(sel_s))
+                t0 = t1 = t2 = None
+            else:
+                t0 = tm.mark(sel_s) if tm and tm.wants("score_select") else None
+                pi.score_select(l, q[l], b.digest, self.ctx_len, b.sel_blocks, b.sel_count, b.scores, stream=sel_s)
+                t1 = tm.mark(sel_s) if tm and (tm.wants("score_select") or tm.wants("diff")) else None
+                pi.diff_misses(l, step, self.ctx_len, b.sel_blocks, b.sel_count, b.block_table, b.slot_block,
+                               b.slot_stamp, b.sel_slots, b.recall_list, b.recall_count, stream=sel_s)
+                t2 = tm.mark(sel_s) if tm and tm.wants("diff") else None
             if overlapped:
                 evd.record(sel_s)
                 rec_s.wait_event(evd)

@@ -141,7 +141,8 @@ def check_near_tie(sel_gpu: set, sel_ref: set, sc: np.ndarray, k_mid: int, cfg, 
         assert abs(sc[b] - tau) <= NEAR_TIE_REL * max(abs(sc[b]), abs(tau)), (b, sc[b], tau)
 
 
-def run_and_compare(case: Case, steps: int, layer: int = 0, overlapped: bool = False, pi_kwargs=None) -> dict:
+def run_and_compare(case: Case, steps: int, layer: int = 0, overlapped: bool = False, pi_kwargs=None,
+                    fused: bool = True) -> dict:
     """The whole path for `steps` decode steps of one layer, checked stage by stage.
     Returns summary statistics."""
     from paper_2609_34555_b200 import PulseInfer
@@ -171,9 +172,9 @@ def run_and_compare(case: Case, steps: int, layer: int = 0, overlapped: bool = F
         q_d = case.q[t].to(dev)
         qb = oracle.bits(case.q[t])
         if overlapped:
-            path.layer_step_overlapped(layer, step, buf, q_d, ctx_d, case.kv, out_d, lse_d)
+            path.layer_step_overlapped(layer, step, buf, q_d, ctx_d, case.kv, out_d, lse_d, fused=fused)
         else:
-            path.layer_step(layer, step, buf, q_d, ctx_d, case.kv, out_d, lse_d)
+            path.layer_step(layer, step, buf, q_d, ctx_d, case.kv, out_d, lse_d, fused=fused)
         torch.cuda.synchronize()
         st = pi.status()
         assert st[0] == 0, f"device status {st}"
@@ -219,7 +220,7 @@ def run_and_compare(case: Case, steps: int, layer: int = 0, overlapped: bool = F
 
 def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, settle_cold: bool = True,
                         append: bool = False, ctx_start: int = 0, paged: bool = False, pi_kwargs=None,
-                        return_out: bool = False) -> dict:
+                        return_out: bool = False, fused: bool = True) -> dict:
     """The bench's launch configuration (DecodeSession: whole batch per call, every layer,
     three-stream pipeline) at a full-size shape; the oracle follows only `sample_seqs`, which is
     enough because sequences are independent.  Inputs are generated on the GPU and handed to the
@@ -229,7 +230,8 @@ def run_session_sampled(cfg, steps: int, sample_seqs, overlapped: bool = True, s
 
     dev = torch.device("cuda:0")
     pi = PulseInfer.from_workload(cfg, **(pi_kwargs or {}))
-    sess = DecodeSession(pi, cfg.batch, cfg.n_layers, keep_scores=True, paged=paged, page_seed=cfg.seed + 5)
+    sess = DecodeSession(pi, cfg.batch, cfg.n_layers, keep_scores=True, paged=paged, page_seed=cfg.seed + 5,
+                         fused_select_diff=fused)
     ctx_now = ctx_start or cfg.ctx                     # runs that append start short of the full context
     sess.ctx_len.fill_(ctx_now)
     short = cfg.replace(ctx=ctx_now)

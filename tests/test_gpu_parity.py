@@ -22,6 +22,53 @@ def test_tiny_ragged_batch_multi_step():
     assert sum(stats["misses"]) > 0
 
 
+@pytest.mark.parametrize("fused", [False, True])
+def test_selection_and_diff_as_two_calls_and_as_one(fused):
+    """The path with pi_score_select + pi_diff_misses, and with pi_score_select_diff, against the oracle:
+    ragged batch, cold pool (many misses: the ranking path of the victim choice), several steps."""
+    from tests.parity import make_case, run_and_compare
+    cfg = tiny_config(batch=4, ctx=5000, n_q_heads=16, n_kv_heads=4, budget_blocks=48, resident_frac=0.25)
+    case = make_case(cfg, steps=5, ctx_len=np.asarray([5000, 4999, 2100, 330]), fill=0.3)
+    stats = run_and_compare(case, steps=5, fused=fused)
+    assert max(stats["misses"]) > 8 and min(stats["misses"]) <= 8
+
+
+def test_one_launch_equals_two_launches_bit_for_bit():
+    """pi_score_select_diff writes exactly what pi_score_select followed by pi_diff_misses writes."""
+    import paper_2609_34555_b200 as pkg
+    from paper_2609_34555_b200.runner import LayerBuffers
+    from workloads import generate as gen
+    for cfg in (get_config("c2").replace(n_layers=1, batch=5), tiny_config(batch=3, ctx=2000, budget_blocks=32, resident_frac=0.3)):
+        dev = torch.device("cuda:0")
+        pi = pkg.PulseInfer.from_workload(cfg)
+        ctx = torch.full((cfg.batch,), cfg.ctx, dtype=torch.int32, device=dev)
+        ctx[-1] = cfg.ctx // 2 + 3
+        q = gen.make_queries(cfg, 0, 4, ar1=0.8).to(dev)
+        res = torch.from_numpy(gen.initial_resident(cfg.replace(ctx=int(ctx[-1])), 0)[:, :cfg.pool_slots]).to(dev)
+        res = torch.nn.functional.pad(res, (0, cfg.pool_slots - res.shape[1]), value=-1).contiguous()
+        digest = torch.randn((cfg.batch, cfg.n_blocks, 2, 128), generator=torch.Generator().manual_seed(3)).to(torch.bfloat16).to(dev)
+        bufs = [LayerBuffers(pi, cfg.batch, dev, keep_scores=True) for _ in range(2)]
+        for b in bufs:
+            b.digest.copy_(digest)
+            pi.table_init(res, b.block_table, b.slot_block, b.slot_stamp)
+        for step in range(1, 5):
+            a, b = bufs
+            pi.score_select(0, q[step - 1], a.digest, ctx, a.sel_blocks, a.sel_count, a.scores)
+            pi.diff_misses(0, step, ctx, a.sel_blocks, a.sel_count, a.block_table, a.slot_block, a.slot_stamp,
+                           a.sel_slots, a.recall_list, a.recall_count)
+            pi.score_select_diff(0, step, q[step - 1], b.digest, ctx, b.sel_blocks, b.sel_count, b.block_table,
+                                 b.slot_block, b.slot_stamp, b.sel_slots, b.recall_list, b.recall_count, scores=b.scores)
+            torch.cuda.synchronize()
+            assert pi.status()[0] == 0, pi.status()
+            for name in ("scores", "sel_blocks", "sel_count", "block_table", "slot_block", "slot_stamp", "sel_slots", "recall_count"):
+                assert torch.equal(getattr(a, name), getattr(b, name)), (step, name)
+            n = a.recall_count.cpu().numpy()
+            for s_ in range(cfg.batch):
+                assert torch.equal(a.recall_list[s_, :n[s_]], b.recall_list[s_, :n[s_]]), (step, s_)
+            assert int(a.recall_count.sum()) > 0 or step > 1
+        pi.close()
+
+
 def test_config1_planted_query():
     from tests.parity import make_case, run_and_compare
     cfg = get_config("c1")
@@ -412,7 +459,7 @@ def test_random_shapes(seed):
     lens = [int(rng.integers(1, cfg.ctx + 1)) for _ in range(batch)]
     lens[0] = cfg.ctx
     case = make_case(cfg, steps=3, ctx_len=np.asarray(lens), fill=float(rng.choice([0.0, 0.5, 1.0])))
-    run_and_compare(case, steps=3, overlapped=bool(seed % 2))
+    run_and_compare(case, steps=3, overlapped=bool(seed % 2), fused=bool((seed // 2) % 2))
 
 
 def test_pipelined_session_with_append_on_two_layers():
