@@ -301,6 +301,9 @@ int pi_build_digests_all(pi_ctx* ctx, int batch, const void* kv, int64_t kv_seq_
 int pi_table_init(pi_ctx* ctx, int batch, const int32_t* resident_dev, int32_t* block_table_dev,
                   int32_t* slot_block_dev, uint32_t* slot_stamp_dev, void* stream);
 int pi_h2d_copy_ms(const void* host_pinned, void* dev, int64_t bytes, int reps, float* best_ms);
+/* Launches a kernel that does nothing (n_ctas x n_threads): timed between two events it gives the
+ * floor under every per-call time of this library on the box at hand (measurement helper). */
+int pi_empty_launch(int n_ctas, int n_threads, void* stream);
 
 /* Sticky device status.  out[0] = first PI_ERR_* code seen by a kernel (0 = none),
  * out[1] = stage (1 score/select, 2 diff, 3 recall, 4 attention, 5 append), out[2..4] = sequence

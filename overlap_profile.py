@@ -1,7 +1,7 @@
 """Overlap-depth profile on the GPU (Sec. 4.3.2 of the paper): how many layers of the normal batch
 fit into the recall I/O of one offload-batch layer, on a grid of batch sizes (B_o, B_n).
 
-    python -m paper_2609_34555_b200.overlap_profile [--out FILE]
+    python overlap_profile.py [--out FILE]
 
 t_io(B_o)    time of selection + diff + recall of one layer for B_o offloaded sequences of the
              Llama-3-8B-shaped workload (32K context, 2048-token budget, settled hot set), measured
@@ -26,7 +26,7 @@ from pathlib import Path
 import numpy as np
 import torch
 
-sys.path.insert(0, str(Path(__file__).resolve().parent.parent))
+sys.path.insert(0, str(Path(__file__).resolve().parent))
 
 from paper_2609_34555_b200 import PulseInfer  # noqa: E402
 from paper_2609_34555_b200.ioaa import OverlapDepthGrid, ioaa_admit  # noqa: E402

@@ -4,4 +4,4 @@ score -> top-k select -> miss diff -> gather-scatter recall -> sparse GQA attent
 The work is done by the CUDA library built from csrc/ behind the C ABI declared in
 include/pulseinfer.h; `binding` is its ctypes front end.
 """
-from .binding import PulseInfer, PiError, score_select_noalloc, load_library, h2d_copy_ms, strerror, EXPORTS  # noqa: F401
+from .binding import PulseInfer, PiError, score_select_noalloc, load_library, h2d_copy_ms, empty_launch, strerror, EXPORTS  # noqa: F401

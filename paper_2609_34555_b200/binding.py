@@ -23,7 +23,7 @@ ERR_NAMES = {
 EXTENT_DTYPE = torch.int32      # a pi_extent is four int32: src_unit, dst_unit, n_units, units_before
 
 EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_score_select_diff", "pi_score_select_diff_devstep", "pi_score_select_noalloc", "pi_score_select_strategy", "pi_diff_misses", "pi_diff_misses_devstep", "pi_recall_gather_scatter",
-           "pi_recall_gather_scatter_paged", "pi_sparse_decode_attn", "pi_sparse_decode_attn_headwise", "pi_append_kv", "pi_append_kv_paged", "pi_append_kv_devstep", "pi_build_digests", "pi_build_digests_all", "pi_table_init", "pi_h2d_copy_ms",
+           "pi_recall_gather_scatter_paged", "pi_sparse_decode_attn", "pi_sparse_decode_attn_headwise", "pi_append_kv", "pi_append_kv_paged", "pi_append_kv_devstep", "pi_build_digests", "pi_build_digests_all", "pi_table_init", "pi_h2d_copy_ms", "pi_empty_launch",
            "pi_get_status", "pi_get_stats", "pi_clear_status", "pi_strerror"]
 
 
@@ -77,6 +77,7 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.pi_build_digests.argtypes = [c_void_p, c_int, c_int, vp, c_int64, i32p, vp, vp]
     lib.pi_table_init.argtypes = [c_void_p, c_int, i32p, i32p, i32p, u32p, vp]
     lib.pi_h2d_copy_ms.argtypes = [vp, vp, c_int64, c_int, POINTER(c_float)]
+    lib.pi_empty_launch.argtypes = [c_int, c_int, vp]
     lib.pi_get_status.argtypes = [c_void_p, POINTER(c_int32 * 8)]
     lib.pi_get_stats.argtypes = [c_void_p, POINTER(c_int64 * 4), c_int]
     lib.pi_clear_status.argtypes = [c_void_p]
@@ -119,6 +120,11 @@ def h2d_copy_ms(host_pinned: torch.Tensor, dev: torch.Tensor, reps: int = 10) ->
     ms = c_float(0)
     _check("pi_h2d_copy_ms", load_library().pi_h2d_copy_ms(host_pinned.data_ptr(), dev.data_ptr(), nbytes, reps, ctypes.byref(ms)))
     return float(ms.value)
+
+
+def empty_launch(n_ctas: int = 128, n_threads: int = 256, stream=None) -> None:
+    """A kernel that does nothing: between two events it measures the launch floor of the box."""
+    _check("pi_empty_launch", load_library().pi_empty_launch(n_ctas, n_threads, _stream(stream)))
 
 
 def score_select_noalloc(q, digest, ctx_len, sel_blocks, sel_count, *, n_kv_heads: int, block_tokens: int,

@@ -100,3 +100,15 @@ int pi_launch_table_init(pi_ctx* c, int batch, const int32_t* resident, int32_t*
     PI_CUDA_TRY(cudaGetLastError());
     return PI_OK;
 }
+
+// A kernel that does nothing, for the measurement of the launch floor.
+namespace {
+__global__ void empty_kernel() {}
+}  // namespace
+
+extern "C" int pi_empty_launch(int n_ctas, int n_threads, void* stream) {
+    if (n_ctas < 1 || n_threads < 1 || n_threads > 1024) return PI_ERR_INVALID_ARG;
+    empty_kernel<<<n_ctas, n_threads, 0, static_cast<cudaStream_t>(stream)>>>();
+    PI_CUDA_TRY(cudaGetLastError());
+    return PI_OK;
+}

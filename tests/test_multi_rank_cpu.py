@@ -65,3 +65,22 @@ def test_cpulist_parser_and_numa_binding_falls_back_quietly():
     before = os.sched_getaffinity(0)
     assert bench.bind_near_gpu(0) is None            # no GPU here: a placement hint must never raise
     assert os.sched_getaffinity(0) == before
+
+
+def test_gpus_flag_starts_the_ranks_itself_when_no_launcher_set_the_environment():
+    """`bench.py --gpus 2` with no WORLD_SIZE in the environment must come back as a two-rank job: the
+    script re-executes itself under torch.distributed.run on 127.0.0.1 (checked here without a GPU: the
+    ranks only call the roll, over gloo)."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--gpus", "2", "--launch-check"], env=env,
+                       capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, r.stdout                      # rank 0 alone prints
+    assert lines[0]["n_gpus"] == 2 and lines[0]["ranks"] == [0, 1] and lines[0]["max_ms"] == 2.0
+    # one rank needs no launcher
+    r1 = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--gpus", "1", "--launch-check"], env=env,
+                        capture_output=True, text=True, timeout=300)
+    assert r1.returncode == 0 and json.loads(r1.stdout.strip().splitlines()[-1])["n_gpus"] == 1
