@@ -58,6 +58,11 @@ typedef struct {
     int32_t max_batch, max_blocks;            /* capacities: batch <= max_batch, NB = max_blocks  */
     int32_t recall_ctas;                      /* CTAs per recall launch, 0 = default (5)           */
     int32_t attn_ctas;                        /* CTAs of the attention kernel, 0 = default (#SMs - 20) */
+    int32_t wait_limit_us;                    /* bound of every device-side wait of the attention kernel in microseconds,
+                                                 0 = default (2 000 000); when it runs out the kernel gives up, returns and
+                                                 the status word says PI_ERR_TIMEOUT (stage 4: CTA, first unit, last unit) */
+    int32_t test_hold_producer;               /* TEST ONLY, keep 0: when 1 the loads of every CTA's last tile are never
+                                                 issued, so that the bounded wait above can be seen to run out */
     const int32_t* solo_head;                 /* host [n_layers]: retrieval KV head per layer (copied) */
 } pi_config;
 
@@ -301,6 +306,14 @@ int pi_build_digests_all(pi_ctx* ctx, int batch, const void* kv, int64_t kv_seq_
 int pi_table_init(pi_ctx* ctx, int batch, const int32_t* resident_dev, int32_t* block_table_dev,
                   int32_t* slot_block_dev, uint32_t* slot_stamp_dev, void* stream);
 int pi_h2d_copy_ms(const void* host_pinned, void* dev, int64_t bytes, int reps, float* best_ms);
+/* Middle attention mass (Eq. 2 of the paper: MAM_q = sum over the middle positions of the attention
+ * weights of query head q), from the log-sum-exps of two attention calls over the same queries: all
+ * blocks (lse_all) and the middle blocks only (lse_mid); the mass of a token set is exp(lse_set - lse_all).
+ *   lse_mid_dev, lse_all_dev [batch][Hq] float (in);  mam_q_dev [batch][Hq] float (out);
+ *   mam_kv_dev [Hkv] float (out): mean over the batch and over each KV head's query heads (Sec. 4.4.1:
+ *   the KV head with the highest value is the layer's retrieval head).  Offline profiling helper. */
+int pi_middle_attention_mass(pi_ctx* ctx, int batch, const float* lse_mid_dev, const float* lse_all_dev,
+                             float* mam_q_dev, float* mam_kv_dev, void* stream);
 /* Launches a kernel that does nothing (n_ctas x n_threads): timed between two events it gives the
  * floor under every per-call time of this library on the box at hand (measurement helper). */
 int pi_empty_launch(int n_ctas, int n_threads, void* stream);

@@ -23,7 +23,7 @@ ERR_NAMES = {
 EXTENT_DTYPE = torch.int32      # a pi_extent is four int32: src_unit, dst_unit, n_units, units_before
 
 EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_score_select_diff", "pi_score_select_diff_devstep", "pi_score_select_noalloc", "pi_score_select_strategy", "pi_diff_misses", "pi_diff_misses_devstep", "pi_recall_gather_scatter",
-           "pi_recall_gather_scatter_paged", "pi_sparse_decode_attn", "pi_sparse_decode_attn_headwise", "pi_append_kv", "pi_append_kv_paged", "pi_append_kv_devstep", "pi_build_digests", "pi_build_digests_all", "pi_table_init", "pi_h2d_copy_ms", "pi_empty_launch",
+           "pi_recall_gather_scatter_paged", "pi_sparse_decode_attn", "pi_sparse_decode_attn_headwise", "pi_append_kv", "pi_append_kv_paged", "pi_append_kv_devstep", "pi_build_digests", "pi_build_digests_all", "pi_table_init", "pi_h2d_copy_ms", "pi_empty_launch", "pi_middle_attention_mass",
            "pi_get_status", "pi_get_stats", "pi_clear_status", "pi_strerror"]
 
 
@@ -32,7 +32,7 @@ class PiConfig(ctypes.Structure):
                 ("block_tokens", c_int32), ("budget_blocks", c_int32), ("n_sink_blocks", c_int32),
                 ("n_local_blocks", c_int32), ("pool_slots", c_int32), ("max_batch", c_int32),
                 ("max_blocks", c_int32), ("recall_ctas", c_int32), ("attn_ctas", c_int32),
-                ("solo_head", POINTER(c_int32))]
+                ("wait_limit_us", c_int32), ("test_hold_producer", c_int32), ("solo_head", POINTER(c_int32))]
 
 
 class PiError(RuntimeError):
@@ -78,6 +78,7 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.pi_table_init.argtypes = [c_void_p, c_int, i32p, i32p, i32p, u32p, vp]
     lib.pi_h2d_copy_ms.argtypes = [vp, vp, c_int64, c_int, POINTER(c_float)]
     lib.pi_empty_launch.argtypes = [c_int, c_int, vp]
+    lib.pi_middle_attention_mass.argtypes = [c_void_p, c_int, vp, vp, vp, vp, vp]
     lib.pi_get_status.argtypes = [c_void_p, POINTER(c_int32 * 8)]
     lib.pi_get_stats.argtypes = [c_void_p, POINTER(c_int64 * 4), c_int]
     lib.pi_clear_status.argtypes = [c_void_p]
@@ -149,13 +150,15 @@ class PulseInfer:
 
     def __init__(self, *, n_layers: int, n_q_heads: int, n_kv_heads: int, block_tokens: int, budget_blocks: int,
                  n_sink_blocks: int, n_local_blocks: int, pool_slots: int, max_batch: int, max_blocks: int,
-                 solo_head: Sequence[int], head_dim: int = 128, recall_ctas: int = 0, attn_ctas: int = 0):
+                 solo_head: Sequence[int], head_dim: int = 128, recall_ctas: int = 0, attn_ctas: int = 0,
+                 wait_limit_us: int = 0, test_hold_producer: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2609_34555_b200 needs a CUDA device; there is no CPU path")
         self._lib = load_library()
         heads = (c_int32 * n_layers)(*[int(h) for h in solo_head])
         self.cfg = PiConfig(n_layers, n_q_heads, n_kv_heads, head_dim, block_tokens, budget_blocks, n_sink_blocks,
-                            n_local_blocks, pool_slots, max_batch, max_blocks, recall_ctas, attn_ctas, heads)
+                            n_local_blocks, pool_slots, max_batch, max_blocks, recall_ctas, attn_ctas, wait_limit_us,
+                            test_hold_producer, heads)
         self._ctx = c_void_p()
         _check("pi_create", self._lib.pi_create(ctypes.byref(self.cfg), ctypes.byref(self._ctx)))
         self.frag_bytes = block_tokens * head_dim * 2 * 2
@@ -338,6 +341,13 @@ class PulseInfer:
         _check("pi_table_init", self._lib.pi_table_init(
             self._ctx, batch, _dev(resident, torch.int32, "resident"), _dev(block_table, torch.int32, "block_table"),
             _dev(slot_block, torch.int32, "slot_block"), _dev(slot_stamp, torch.int32, "slot_stamp"), _stream(stream)))
+
+    def middle_attention_mass(self, lse_mid, lse_all, mam_q, mam_kv, stream=None) -> None:
+        """Eq. 2 from two log-sum-exps: mam_q [batch][Hq] = exp(lse_mid - lse_all), mam_kv [Hkv] = its mean
+        over the batch and over each KV head's query heads."""
+        _check("pi_middle_attention_mass", self._lib.pi_middle_attention_mass(
+            self._ctx, lse_all.shape[0], _dev(lse_mid, torch.float32, "lse_mid"), _dev(lse_all, torch.float32, "lse_all"),
+            _dev(mam_q, torch.float32, "mam_q"), _dev(mam_kv, torch.float32, "mam_kv"), _stream(stream)))
 
     def status(self) -> list[int]:
         out = (c_int32 * 8)()

@@ -23,7 +23,8 @@ int check_config(const pi_config* c) {
     if (c->budget_blocks > 4096) return PI_ERR_UNSUPPORTED_DIM;
     if (c->pool_slots < c->budget_blocks) return PI_ERR_POOL_TOO_SMALL;
     if (c->pool_slots > 8192) return PI_ERR_UNSUPPORTED_DIM;
-    if (c->recall_ctas < 0 || c->attn_ctas < 0) return PI_ERR_INVALID_ARG;
+    if (c->recall_ctas < 0 || c->attn_ctas < 0 || c->wait_limit_us < 0) return PI_ERR_INVALID_ARG;
+    if (c->test_hold_producer != 0 && c->test_hold_producer != 1) return PI_ERR_INVALID_ARG;
     for (int l = 0; l < c->n_layers; ++l)
         if (c->solo_head[l] < 0 || c->solo_head[l] >= c->n_kv_heads) return PI_ERR_INVALID_ARG;
     return PI_OK;
@@ -65,6 +66,9 @@ extern "C" int pi_create(const pi_config* cfg, pi_ctx** out) {
     // streams saturate the host link of a B200 and cover each other's fixed costs; one launch alone
     // still reaches 0.97 of what ten CTAs do, and more requests in flight only queue up
     c->recall_ctas = cfg->recall_ctas > 0 ? cfg->recall_ctas : 5;
+    // a wait that lasts this long is a failure: the kernel gives up and reports (default: two seconds)
+    c->wait_limit_cycles = static_cast<long long>(cfg->wait_limit_us > 0 ? cfg->wait_limit_us : 2000000) *
+                           (prop.clockRate > 0 ? prop.clockRate : 1000000) / 1000;
 
     const size_t nb = static_cast<size_t>(cfg->max_batch);
     const size_t n_part = static_cast<size_t>(c->attn_ctas) + nb;

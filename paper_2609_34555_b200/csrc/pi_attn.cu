@@ -22,7 +22,6 @@ constexpr int ATTN_MAX_STAGES = 8;
 constexpr int ATTN_META_UNITS = 1024;              // units per CTA whose metadata is staged in shared memory
 constexpr int ATTN_SMEM_BUDGET = 196 * 1024;       // ring bytes
 constexpr int MERGE_BATCH = 12;                    // partial outputs a lane of the merge kernel has in flight
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s: a wait this long is a failure
 
 struct AttnParams {
     const __nv_bfloat16* q;
@@ -38,6 +37,8 @@ struct AttnParams {
     pi_status_ref st;
     int batch, Hq, Hkv, G, B, K, C, stages;
     int headwise;                 // 1: sel_slots / sel_blocks are [batch][Hkv][K], sel_count [batch][Hkv]
+    int hold_last;                // test only: the producer never issues the loads of its CTA's last unit
+    long long wait_cycles;        // bound of every wait on a barrier
     float scale_log2;
 };
 
@@ -76,7 +77,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait: gives up when another warp raised `abort` or the cycle limit passes.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort, long long limit) {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
@@ -84,7 +85,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         for (int i = 0; i < 64; ++i)
             if (mbar_try(bar, parity)) return true;
         if (*abort) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort = 1; return false; }
+        if (clock64() - t0 > limit) { *abort = 1; return false; }
     }
 }
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
@@ -352,7 +353,8 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
             for (int u = u0, it = 0; u < u1; ++u, ++it) {
                 while (u >= s_pref[seq + 1]) ++seq;
                 const int st = it % p.stages, round = it / p.stages;
-                if (round > 0 && !mbar_wait(bar_empty + 8 * st, (round - 1) & 1, s_abort)) break;
+                if (round > 0 && !mbar_wait(bar_empty + 8 * st, (round - 1) & 1, s_abort, p.wait_cycles)) break;
+                if (p.hold_last && u == u1 - 1) break;           // (test only) the consumers' wait for this unit runs out
                 const uint32_t dst = ring + st * stage_bytes;
                 // valid-token counts are written before the arrive below, which publishes them
                 if (HW) {
@@ -413,7 +415,7 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
         }
       for (; u < seg_end; ++u, ++it) {
         const int st = it % p.stages;
-        if (!mbar_wait(bar_full + 8 * st, (it / p.stages) & 1, s_abort)) { alive = false; break; }
+        if (!mbar_wait(bar_full + 8 * st, (it / p.stages) & 1, s_abort, p.wait_cycles)) { alive = false; break; }
         const int nvalid = s_nvalid[st * 8 + (HW ? h : 0)];
         const uint32_t base = ring + st * stage_bytes;
 
@@ -573,6 +575,8 @@ int pi_launch_attn(pi_ctx* c, int batch, const void* q, const void* pool, const 
     p.batch = batch; p.Hq = cfg.n_q_heads; p.Hkv = cfg.n_kv_heads; p.G = cfg.n_q_heads / cfg.n_kv_heads;
     p.B = cfg.block_tokens; p.K = cfg.budget_blocks; p.C = cfg.pool_slots;
     p.headwise = headwise ? 1 : 0;
+    p.hold_last = cfg.test_hold_producer;
+    p.wait_cycles = c->wait_limit_cycles;
     const int stage_bytes = cfg.n_kv_heads * 8192;
     int stages = ATTN_SMEM_BUDGET / stage_bytes;
     if (stages > ATTN_MAX_STAGES) stages = ATTN_MAX_STAGES;

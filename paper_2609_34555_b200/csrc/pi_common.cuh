@@ -58,6 +58,7 @@ struct pi_ctx {
     float* attn_part_o;          // [attn_ctas + max_batch][Hq][D]
     float* attn_part_ml;         // [attn_ctas + max_batch][Hq][2]
     int attn_ctas, recall_ctas;
+    long long wait_limit_cycles; // bound of the attention kernel's waits, in SM cycles
     unsigned long long* stats_dev; // [4]: sequences diffed, selected blocks, missing blocks, extents
     // status: device flag (first writer wins) + pinned mirror the kernels fill in
     int* status_flag_dev;

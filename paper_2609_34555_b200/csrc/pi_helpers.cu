@@ -112,3 +112,29 @@ extern "C" int pi_empty_launch(int n_ctas, int n_threads, void* stream) {
     PI_CUDA_TRY(cudaGetLastError());
     return PI_OK;
 }
+
+// Last step of Eq. 2: mass of the middle tokens per query head, and its mean per KV head.
+namespace {
+__global__ void mam_kernel(const float* lse_mid, const float* lse_all, float* mam_q, float* mam_kv, int batch, int Hq, int G) {
+    __shared__ float acc[16];
+    if (threadIdx.x < 16) acc[threadIdx.x] = 0.f;
+    __syncthreads();
+    for (int i = threadIdx.x; i < batch * Hq; i += blockDim.x) {
+        const float a = lse_all[i], m = lse_mid[i];
+        const float v = (m == -INFINITY || a == -INFINITY) ? 0.f : expf(m - a);
+        mam_q[i] = v;
+        atomicAdd(&acc[(i % Hq) / G], v);
+    }
+    __syncthreads();
+    if (threadIdx.x < Hq / G) mam_kv[threadIdx.x] = acc[threadIdx.x] / static_cast<float>(batch * G);
+}
+}  // namespace
+
+extern "C" int pi_middle_attention_mass(pi_ctx* ctx, int batch, const float* lse_mid_dev, const float* lse_all_dev,
+                                        float* mam_q_dev, float* mam_kv_dev, void* stream) {
+    if (!ctx || batch < 1 || !lse_mid_dev || !lse_all_dev || !mam_q_dev || !mam_kv_dev) return PI_ERR_INVALID_ARG;
+    const int Hq = ctx->cfg.n_q_heads, G = Hq / ctx->cfg.n_kv_heads;
+    mam_kernel<<<1, 256, 0, static_cast<cudaStream_t>(stream)>>>(lse_mid_dev, lse_all_dev, mam_q_dev, mam_kv_dev, batch, Hq, G);
+    PI_CUDA_TRY(cudaGetLastError());
+    return PI_OK;
+}

@@ -196,9 +196,8 @@ class CudaOffload:
         ev = self.torch.cuda.Event()
         ev.record(self.compute_stream)                    # the layer's query exists once the previous layer is done
         s.side.wait_event(ev)
-        pi.score_select(l, q, b.digest, s.ctx_len, b.sel_blocks, b.sel_count, None, stream=s.side)
-        pi.diff_misses(l, self.step, s.ctx_len, b.sel_blocks, b.sel_count, b.block_table, b.slot_block, b.slot_stamp,
-                       b.sel_slots, b.recall_list, b.recall_count, stream=s.side)
+        pi.score_select_diff(l, self.step, q, b.digest, s.ctx_len, b.sel_blocks, b.sel_count, b.block_table, b.slot_block,
+                             b.slot_stamp, b.sel_slots, b.recall_list, b.recall_count, stream=s.side)
         d = self.torch.cuda.Event(); d.record(s.side); s.side2.wait_event(d)
         pi.recall_gather_scatter(l, s.host_region(l), b.pool, b.recall_list, b.recall_count, stream=s.side2)
         io = self.torch.cuda.Event(enable_timing=True)

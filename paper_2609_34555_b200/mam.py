@@ -2,9 +2,10 @@
 
 MAM_q = sum over middle positions i of the attention weight A_q(i); the MAM of a KV head is the
 mean over the query heads that GQA maps to it; the KV head with the highest MAM of a layer is
-its retrieval ("SoloHead") head (Sec. 4.4.1).  No new kernel is needed: with lse_S the
-log-sum-exp of the logits over a token set S,  sum_{i in S} A(i) = exp(lse_S - lse_all), so two
-calls of pi_sparse_decode_attn (all blocks, middle blocks only) give the mass.  "Middle" is
+its retrieval ("SoloHead") head (Sec. 4.4.1).  With lse_S the log-sum-exp of the logits over a
+token set S,  sum_{i in S} A(i) = exp(lse_S - lse_all): two calls of pi_sparse_decode_attn (all
+blocks, middle blocks only) and pi_middle_attention_mass give the mass and its per-KV-head mean;
+picking the arg-max of Hkv numbers is left to the host.  "Middle" is
 block-granular here, like the path's sink and local blocks.  The sample sequences must be fully
 resident in the pool (slot i = block i); this is an offline profiling helper, not a hot call.
 """
@@ -15,9 +16,11 @@ import torch
 from .binding import PulseInfer
 
 
-def middle_attention_mass(pi: PulseInfer, layer: int, q: torch.Tensor, pool: torch.Tensor, ctx_len: torch.Tensor) -> torch.Tensor:
+def middle_attention_mass(pi: PulseInfer, layer: int, q: torch.Tensor, pool: torch.Tensor, ctx_len: torch.Tensor,
+                          return_kv: bool = False):
     """q [batch][Hq][D] bf16, pool [batch][C >= n_blocks] blocks with slot i = block i.
-    Returns MAM per query head, float32 [batch][Hq]."""
+    Returns MAM per query head, float32 [batch][Hq]; with return_kv also the per-KV-head mean [Hkv]
+    (both from pi_middle_attention_mass)."""
     c = pi.cfg
     batch, dev = q.shape[0], q.device
     K, B = c.budget_blocks, c.block_tokens
@@ -38,11 +41,15 @@ def middle_attention_mass(pi: PulseInfer, layer: int, q: torch.Tensor, pool: tor
     mcnt = (hi - lo).contiguous()
     msel = torch.where(idx < mcnt[:, None], idx + lo[:, None], torch.full_like(idx, -1)).contiguous()
     pi.sparse_decode_attn(layer, q, pool, msel, msel, mcnt, ctx_len, out, lse_mid)
-    return torch.exp(lse_mid - lse_all)
+    mam_q = torch.empty_like(lse_all)
+    mam_kv = torch.empty((c.n_kv_heads,), dtype=torch.float32, device=dev)
+    pi.middle_attention_mass(lse_mid, lse_all, mam_q, mam_kv)
+    return (mam_q, mam_kv) if return_kv else mam_q
 
 
 def kv_head_mam(mam_q: torch.Tensor, n_kv_heads: int) -> torch.Tensor:
-    """Mean over samples and over each KV head's query heads: [Hkv]."""
+    """Mean over samples and over each KV head's query heads: [Hkv] (host-side regrouping of masses
+    that pi_middle_attention_mass has computed, for samples collected over several calls)."""
     batch, Hq = mam_q.shape
     return mam_q.view(batch, n_kv_heads, Hq // n_kv_heads).mean(dim=(0, 2))
 

@@ -1,0 +1,105 @@
+"""The interruptible layer-wise scheduler (Sec. 4.2.1 - 4.2.2 of the paper) over its CUDA back end: the
+offload batch advances layer by layer through selection + diff -> recall -> attention while the normal
+batch fills the recall waits; all three ways of noticing that a recall has landed must leave the offload
+batch with exactly the results of the plain serial decode steps, and the semi-synchronous one must hand
+the GPU back to the offload batch sooner than the other two."""
+import statistics
+
+import numpy as np
+import pytest
+import torch
+
+from workloads import generate as gen, get_config, tiny_config
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _need_gpu():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+
+
+def _offload_session(cfg, dev):
+    from paper_2609_34555_b200 import PulseInfer
+    from paper_2609_34555_b200.runner import DecodeSession
+    pi = PulseInfer.from_workload(cfg, recall_ctas=10)          # one recall in flight at a time here
+    sess = DecodeSession(pi, cfg.batch, cfg.n_layers)
+    sess.ctx_len.fill_(cfg.ctx)
+    for l in range(cfg.n_layers):
+        sess.load_layer(l, gen.make_kv(cfg, l, device=dev), torch.from_numpy(gen.initial_resident(cfg, l)).to(dev))
+    torch.cuda.synchronize()
+    return pi, sess
+
+
+def _state(sess):
+    return [(b.block_table.clone(), b.slot_block.clone(), b.slot_stamp.clone(), b.sel_blocks.clone(), b.sel_slots.clone(),
+             b.pool.clone()) for b in sess.bufs]
+
+
+def test_three_detection_modes_on_the_gpu_equal_the_serial_steps_and_order_as_described():
+    from paper_2609_34555_b200 import PulseInfer
+    from paper_2609_34555_b200.irq import MODES, CudaNormal, CudaOffload, IrqScheduler
+    from paper_2609_34555_b200.runner import LayerBuffers
+    dev = torch.device("cuda:0")
+    cfg = get_config("c2").replace(n_layers=3, batch=4, ctx=16384, budget_blocks=96, resident_frac=0.2, seed=11)
+    steps = 6
+    q_all = torch.stack([gen.make_queries(cfg, l, steps, device=dev, ar1=0.8) for l in range(cfg.n_layers)], 1).contiguous()
+
+    # the plain serial decode steps from the same start
+    pi_r, ref = _offload_session(cfg, dev)
+    for t in range(steps):
+        ref.decode_step(q_all[t], overlapped=False)
+    torch.cuda.synchronize()
+    assert pi_r.status()[0] == 0
+    want_out, want_state = ref.out.clone(), _state(ref)
+    misses = pi_r.stats()["missing_blocks"]
+    assert misses > 0
+    pi_r.close()
+    del ref
+
+    # the normal batch: short requests whose KV is all on the GPU (every block selected, slot i = block i)
+    ncfg = tiny_config(batch=32, ctx=2048, n_q_heads=32, n_kv_heads=8, budget_blocks=128, resident_frac=1.0, n_layers=1)
+    npi = PulseInfer.from_workload(ncfg)
+    nbuf = LayerBuffers(npi, ncfg.batch, dev)
+    nbuf.pool.copy_(torch.randn(nbuf.pool.shape[:2] + (1,) * 4, device=dev).to(torch.bfloat16).expand_as(nbuf.pool))
+    ident = torch.arange(ncfg.n_blocks, dtype=torch.int32, device=dev)[None, :].expand(ncfg.batch, -1).contiguous()
+    nbuf.sel_slots.copy_(ident); nbuf.sel_blocks.copy_(ident); nbuf.sel_count.fill_(ncfg.n_blocks)
+    nq = torch.randn((ncfg.batch, ncfg.n_q_heads, 128), device=dev).to(torch.bfloat16)
+    nctx = torch.full((ncfg.batch,), ncfg.ctx, dtype=torch.int32, device=dev)
+    nout = torch.zeros_like(nq)
+    # FFN stand-ins (plumbing, 8B-shaped): they make a normal layer last long enough to tell the modes apart
+    w1 = torch.randn((4096, 14336), device=dev, dtype=torch.bfloat16) * 0.01
+    w2 = torch.randn((14336, 4096), device=dev, dtype=torch.bfloat16) * 0.01
+    xn = torch.randn((256, 4096), device=dev, dtype=torch.bfloat16)
+    xo = torch.randn((cfg.batch, 4096), device=dev, dtype=torch.bfloat16)
+    ffn_n = lambda: torch.matmul(torch.matmul(xn, w1), w2)
+    ffn_o = lambda: torch.matmul(torch.matmul(xo, w1), w2)
+
+    delays = {}
+    for mode in MODES:
+        pi, sess = _offload_session(cfg, dev)
+        off = CudaOffload(sess, q_all, ffn_o)
+        nor = CudaNormal(npi, nbuf, nq, nctx, nout, ffn_n, 32)
+        rep = IrqScheduler(off, nor, mode).run(steps * cfg.n_layers)
+        torch.cuda.synchronize()
+        assert pi.status()[0] == 0 and npi.status()[0] == 0, (pi.status(), npi.status())
+        # (i) the offload batch ends exactly where the serial steps end
+        assert torch.equal(sess.out.view(torch.int16), want_out.view(torch.int16)), f"{mode}: outputs"
+        for l, (got, want) in enumerate(zip(_state(sess), want_state)):
+            for g, w, name in zip(got, want, ("block_table", "slot_block", "slot_stamp", "sel_blocks", "sel_slots", "pool")):
+                assert torch.equal(g.view(torch.int16) if g.dtype == torch.bfloat16 else g,
+                                   w.view(torch.int16) if w.dtype == torch.bfloat16 else w), f"{mode}: layer {l} {name}"
+        assert pi.stats()["missing_blocks"] == misses
+        # (ii) book-keeping of the scheduler
+        assert rep.offload_layers == steps * cfg.n_layers == len(rep.depths)
+        assert rep.normal_layers == sum(rep.depths) and rep.normal_layers > 0
+        assert len(rep.resume_delay_us) == rep.offload_layers
+        delays[mode] = statistics.fmean(rep.resume_delay_us)
+        pi.close()
+        del sess
+    npi.close()
+    print("mean resume delay (us):", {k: round(v, 1) for k, v in delays.items()})
+    # (iii) semi-synchronous detection hands the GPU back sooner than waiting for whole layers (sync) and
+    # sooner than never waiting at all (async: the layers already queued run first)
+    assert delays["semi"] < delays["async"] and delays["semi"] < delays["sync"], delays

@@ -282,6 +282,36 @@ def test_sequences_that_no_cta_splits_pipelined_and_repeatable():
     assert torch.equal(outs[0], outs[1])
 
 
+def test_a_bounded_wait_that_runs_out_is_reported_and_nothing_hangs():
+    """A short wait limit and the test-only hold-back of every CTA's last tile: the consumers' wait for that
+    tile runs out, the kernel returns by itself, the status word says PI_ERR_TIMEOUT (stage 4) and the
+    context stays usable: after clearing the status the same shapes run clean on a context without the hook."""
+    import time
+    from tests.parity import make_case, run_and_compare
+    import paper_2609_34555_b200 as pkg
+    from paper_2609_34555_b200.runner import LayerBuffers
+    cfg = tiny_config(batch=2, ctx=2000, n_q_heads=16, n_kv_heads=4, budget_blocks=24, resident_frac=1.0)
+    dev = torch.device("cuda:0")
+    pi = pkg.PulseInfer.from_workload(cfg, wait_limit_us=300, test_hold_producer=1)
+    buf = LayerBuffers(pi, cfg.batch, dev)
+    ident = torch.arange(cfg.budget_blocks, dtype=torch.int32, device=dev)[None, :].expand(cfg.batch, -1).contiguous()
+    buf.sel_slots.copy_(ident); buf.sel_blocks.copy_(ident); buf.sel_count.fill_(cfg.budget_blocks)
+    q = torch.randn((cfg.batch, cfg.n_q_heads, 128), device=dev).to(torch.bfloat16)
+    ctx = torch.full((cfg.batch,), cfg.ctx, dtype=torch.int32, device=dev)
+    out = torch.zeros_like(q)
+    t0 = time.perf_counter()
+    pi.sparse_decode_attn(0, q, buf.pool, buf.sel_slots, buf.sel_blocks, buf.sel_count, ctx, out)
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 5.0                      # gave up after the limit, not after seconds
+    st = pi.status()
+    assert st[0] == -7 and st[1] == 4 and st[3] < st[4], st    # timeout, attention stage, the CTA's unit range
+    pi.clear_status()
+    assert pi.status()[0] == 0
+    pi.close()
+    # the device and the library are fine afterwards
+    run_and_compare(make_case(cfg, steps=2), steps=2)
+
+
 def test_append_then_decode_with_growing_ragged_contexts():
     from tests.parity import run_append_and_compare
     cfg = tiny_config(batch=4, ctx=1200, n_q_heads=16, n_kv_heads=4, budget_blocks=24, resident_frac=0.4)
@@ -317,7 +347,9 @@ def test_middle_attention_mass_and_retrieval_head_choice():
     pool = torch.zeros((cfg.batch, cfg.pool_slots) + tuple(kv.shape[2:]), dtype=torch.bfloat16, device=dev)
     pool[:, :cfg.n_blocks] = kv.to(dev)
     ctx = torch.tensor([1500, 1111, 700], dtype=torch.int32, device=dev)
-    mam = middle_attention_mass(pi, 0, q.to(dev), pool, ctx).cpu().numpy()
+    mam_t, mam_kv = middle_attention_mass(pi, 0, q.to(dev), pool, ctx, return_kv=True)
+    assert torch.allclose(mam_kv.cpu(), kv_head_mam(mam_t.cpu(), cfg.n_kv_heads), rtol=1e-5, atol=1e-7)
+    mam = mam_t.cpu().numpy()
     kvb, qb = oracle.bits(kv), oracle.bits(q)
     for s in range(cfg.batch):
         nb = -(-int(ctx[s]) // cfg.block_tokens)
