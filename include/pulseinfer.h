@@ -58,6 +58,9 @@ typedef struct {
     int32_t max_batch, max_blocks;            /* capacities: batch <= max_batch, NB = max_blocks  */
     int32_t recall_ctas;                      /* CTAs per recall launch, 0 = default (5)           */
     int32_t attn_ctas;                        /* CTAs of the attention kernel, 0 = default (#SMs - 20) */
+    int32_t attn_mode;                        /* split of the attention work: 0 = chosen per call, 1 = flat (all KV heads of a block
+                                                 per tile, sequences cut across CTAs, partials merged by a second kernel),
+                                                 2 = head-major (one (sequence, KV head) per CTA, merged inside the CTA) */
     int32_t wait_limit_us;                    /* bound of every device-side wait of the attention kernel in microseconds,
                                                  0 = default (2 000 000); when it runs out the kernel gives up, returns and
                                                  the status word says PI_ERR_TIMEOUT (stage 4: CTA, first unit, last unit) */

@@ -32,7 +32,7 @@ class PiConfig(ctypes.Structure):
                 ("block_tokens", c_int32), ("budget_blocks", c_int32), ("n_sink_blocks", c_int32),
                 ("n_local_blocks", c_int32), ("pool_slots", c_int32), ("max_batch", c_int32),
                 ("max_blocks", c_int32), ("recall_ctas", c_int32), ("attn_ctas", c_int32),
-                ("wait_limit_us", c_int32), ("test_hold_producer", c_int32), ("solo_head", POINTER(c_int32))]
+                ("attn_mode", c_int32), ("wait_limit_us", c_int32), ("test_hold_producer", c_int32), ("solo_head", POINTER(c_int32))]
 
 
 class PiError(RuntimeError):
@@ -151,13 +151,13 @@ class PulseInfer:
     def __init__(self, *, n_layers: int, n_q_heads: int, n_kv_heads: int, block_tokens: int, budget_blocks: int,
                  n_sink_blocks: int, n_local_blocks: int, pool_slots: int, max_batch: int, max_blocks: int,
                  solo_head: Sequence[int], head_dim: int = 128, recall_ctas: int = 0, attn_ctas: int = 0,
-                 wait_limit_us: int = 0, test_hold_producer: int = 0):
+                 attn_mode: int = 0, wait_limit_us: int = 0, test_hold_producer: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2609_34555_b200 needs a CUDA device; there is no CPU path")
         self._lib = load_library()
         heads = (c_int32 * n_layers)(*[int(h) for h in solo_head])
         self.cfg = PiConfig(n_layers, n_q_heads, n_kv_heads, head_dim, block_tokens, budget_blocks, n_sink_blocks,
-                            n_local_blocks, pool_slots, max_batch, max_blocks, recall_ctas, attn_ctas, wait_limit_us,
+                            n_local_blocks, pool_slots, max_batch, max_blocks, recall_ctas, attn_ctas, attn_mode, wait_limit_us,
                             test_hold_producer, heads)
         self._ctx = c_void_p()
         _check("pi_create", self._lib.pi_create(ctypes.byref(self.cfg), ctypes.byref(self._ctx)))

@@ -14,7 +14,7 @@ CSRC = PKG / "csrc"
 INCLUDE = PKG.parent / "include"
 LIB = PKG / "libpulseinfer_b200.so"
 
-SOURCES = ["pi_api.cu", "pi_score_select.cu", "pi_select_diff.cu", "pi_diff_misses.cu", "pi_recall.cu", "pi_attn.cu",
+SOURCES = ["pi_api.cu", "pi_score_select.cu", "pi_select_diff.cu", "pi_diff_misses.cu", "pi_recall.cu", "pi_attn.cu", "pi_attn_headmajor.cu",
            "pi_helpers.cu", "pi_append.cu"]
 
 

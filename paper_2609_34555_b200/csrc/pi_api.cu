@@ -25,6 +25,7 @@ int check_config(const pi_config* c) {
     if (c->pool_slots > 8192) return PI_ERR_UNSUPPORTED_DIM;
     if (c->recall_ctas < 0 || c->attn_ctas < 0 || c->wait_limit_us < 0) return PI_ERR_INVALID_ARG;
     if (c->test_hold_producer != 0 && c->test_hold_producer != 1) return PI_ERR_INVALID_ARG;
+    if (c->attn_mode < 0 || c->attn_mode > 2) return PI_ERR_INVALID_ARG;
     for (int l = 0; l < c->n_layers; ++l)
         if (c->solo_head[l] < 0 || c->solo_head[l] >= c->n_kv_heads) return PI_ERR_INVALID_ARG;
     return PI_OK;

@@ -127,6 +127,11 @@ int pi_launch_recall(pi_ctx*, int n_lists, int lists_per_seq, const void* host_k
 int pi_launch_attn(pi_ctx*, int batch, const void* q, const void* pool, const int32_t* sel_slots,
                    const int32_t* sel_blocks, const int32_t* sel_count, const int32_t* ctx_len,
                    void* out, float* lse, int headwise, cudaStream_t);
+// head-major form of the attention (one (sequence, KV head) per CTA); `fits` says whether the items fill the grid evenly
+bool pi_attn_headmajor_fits(const pi_ctx*, int batch, int* grid_out, int* items_per_cta_out, int* split_out);
+int pi_launch_attn_headmajor(pi_ctx*, int batch, const void* q, const void* pool, const int32_t* sel_slots,
+                             const int32_t* sel_blocks, const int32_t* sel_count, const int32_t* ctx_len,
+                             void* out, float* lse, int headwise, cudaStream_t);
 int pi_launch_append(pi_ctx*, int h_star, int batch, uint32_t step, const void* k_new, const void* v_new,
                      const int32_t* ctx_len, void* host_kv, int64_t host_stride, void* pool, int32_t* table,
                      int32_t* slot_block, uint32_t* slot_stamp, void* digest, const int32_t* page_table,

@@ -282,7 +282,8 @@ def test_sequences_that_no_cta_splits_pipelined_and_repeatable():
     assert torch.equal(outs[0], outs[1])
 
 
-def test_a_bounded_wait_that_runs_out_is_reported_and_nothing_hangs():
+@pytest.mark.parametrize("mode", [1, 2])
+def test_a_bounded_wait_that_runs_out_is_reported_and_nothing_hangs(mode):
     """A short wait limit and the test-only hold-back of every CTA's last tile: the consumers' wait for that
     tile runs out, the kernel returns by itself, the status word says PI_ERR_TIMEOUT (stage 4) and the
     context stays usable: after clearing the status the same shapes run clean on a context without the hook."""
@@ -292,7 +293,7 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_nothing_hangs():
     from paper_2609_34555_b200.runner import LayerBuffers
     cfg = tiny_config(batch=2, ctx=2000, n_q_heads=16, n_kv_heads=4, budget_blocks=24, resident_frac=1.0)
     dev = torch.device("cuda:0")
-    pi = pkg.PulseInfer.from_workload(cfg, wait_limit_us=300, test_hold_producer=1)
+    pi = pkg.PulseInfer.from_workload(cfg, wait_limit_us=300, test_hold_producer=1, attn_mode=mode)
     buf = LayerBuffers(pi, cfg.batch, dev)
     ident = torch.arange(cfg.budget_blocks, dtype=torch.int32, device=dev)[None, :].expand(cfg.batch, -1).contiguous()
     buf.sel_slots.copy_(ident); buf.sel_blocks.copy_(ident); buf.sel_count.fill_(cfg.budget_blocks)
@@ -304,7 +305,7 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_nothing_hangs():
     torch.cuda.synchronize()
     assert time.perf_counter() - t0 < 5.0                      # gave up after the limit, not after seconds
     st = pi.status()
-    assert st[0] == -7 and st[1] == 4 and st[3] < st[4], st    # timeout, attention stage, the CTA's unit range
+    assert st[0] == -7 and st[1] == 4 and st[3] < st[4], st    # timeout, attention stage, the CTA's units
     pi.clear_status()
     assert pi.status()[0] == 0
     pi.close()
@@ -494,6 +495,45 @@ def test_random_shapes(seed):
     run_and_compare(case, steps=3, overlapped=bool(seed % 2), fused=bool((seed // 2) % 2))
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_random_shapes_with_the_head_major_attention(seed):
+    """The same kind of random small shapes with the attention forced into its head-major form (one
+    (sequence, KV head) per CTA, eight warps sharing the tokens, merge inside the CTA): few items per
+    grid, several items per CTA (attn_ctas below the item count), ragged and empty sequences, G up to 16."""
+    from tests.parity import make_case, run_and_compare
+    rng = np.random.default_rng(2000 + seed)
+    Hkv = int(rng.choice([1, 2, 4, 8]))
+    G = int(rng.choice([1, 2, 4, 8, 16]))
+    B = int(rng.choice([16, 32, 64]))
+    batch = int(rng.integers(1, 6))
+    nb = int(rng.integers(12, 120))
+    sink = int(rng.choice([0, 16]))
+    local = int(rng.choice([0, 128]))
+    pinned = (-(-sink // B) if sink else 0) + (max(1, local // B) if local else 0)
+    K = int(rng.integers(pinned + 1, pinned + 40))
+    cfg = tiny_config(batch=batch, ctx=nb * B - int(rng.integers(0, B)), n_q_heads=Hkv * G, n_kv_heads=Hkv,
+                      block_tokens=B, budget_blocks=K, resident_frac=float(rng.uniform(0.1, 0.9)),
+                      sink_tokens=sink, local_tokens=local, seed=100 + seed)
+    lens = [int(rng.integers(0, cfg.ctx + 1)) for _ in range(batch)]
+    lens[0] = cfg.ctx
+    case = make_case(cfg, steps=3, ctx_len=np.asarray(lens), fill=float(rng.choice([0.0, 0.5, 1.0])))
+    ctas = int(rng.choice([0, 1, 3, 7]))                       # 0: one CTA per item; else several items per CTA
+    run_and_compare(case, steps=3, overlapped=bool(seed % 2), pi_kwargs=dict(attn_mode=2, attn_ctas=ctas))
+
+
+@pytest.mark.parametrize("mode", [1, 2])
+def test_both_attention_forms_on_the_bench_shapes(mode):
+    """Config 2's per-layer shapes (batch 16 x 8 KV heads = 128 items) with the flat and with the head-major
+    attention, pipelined session, oracle on three sequences; two runs of a form give the same bits."""
+    from tests.parity import run_session_sampled
+    cfg = get_config("c2").replace(n_layers=2)
+    outs = []
+    for _ in range(2):
+        st = run_session_sampled(cfg, steps=2, sample_seqs=[0, 9, 15], pi_kwargs=dict(attn_mode=mode), return_out=True)
+        outs.append(st["out"])
+    assert torch.equal(outs[0], outs[1])
+
+
 def test_pipelined_session_with_append_on_two_layers():
     """DecodeSession's three-stream step with a token appended to every layer each step; the
     context crosses a block boundary on the way."""
@@ -602,7 +642,8 @@ def test_double_buffered_host_stepping_matches_plain_stepping():
         assert torch.equal(outs[0][t].view(torch.int16), outs[2][t].view(torch.int16)), f"step {t}, graph replay"
 
 
-def test_headwise_attention_with_unequal_and_empty_head_lists():
+@pytest.mark.parametrize("mode", [1, 2])
+def test_headwise_attention_with_unequal_and_empty_head_lists(mode):
     """Every KV head attends over its own list; lists of one sequence differ in length, one is empty,
     the last block is partial.  Pool slot i holds block i, so slots and blocks coincide."""
     import numpy as np
@@ -614,7 +655,7 @@ def test_headwise_attention_with_unequal_and_empty_head_lists():
     cfg = tiny_config(batch=3, ctx=16 * 37 + 5, n_q_heads=16, n_kv_heads=4, budget_blocks=20, resident_frac=1.0)
     nb, Hkv, K, G = cfg.n_blocks, cfg.n_kv_heads, cfg.budget_blocks, cfg.group
     assert cfg.pool_slots >= nb
-    pi = PulseInfer.from_workload(cfg)
+    pi = PulseInfer.from_workload(cfg, attn_mode=mode)
     kv = gen.make_kv(cfg, 0)
     kvb = oracle.bits(kv)
     pool = torch.zeros((cfg.batch, cfg.pool_slots) + tuple(kv.shape[2:]), dtype=torch.bfloat16)

@@ -36,7 +36,7 @@ def test_error_strings():
 def _cfg(**kw):
     base = dict(n_layers=1, n_q_heads=32, n_kv_heads=8, head_dim=128, block_tokens=16, budget_blocks=64,
                 n_sink_blocks=1, n_local_blocks=8, pool_slots=128, max_batch=4, max_blocks=512,
-                recall_ctas=0, attn_ctas=0, wait_limit_us=0, test_hold_producer=0)
+                recall_ctas=0, attn_ctas=0, attn_mode=0, wait_limit_us=0, test_hold_producer=0)
     base.update(kw)
     heads = (ctypes.c_int32 * base["n_layers"])(*([0] * base["n_layers"]))
     return PiConfig(*[base[f] for f, _ in PiConfig._fields_[:-1]], heads), heads
@@ -45,7 +45,7 @@ def _cfg(**kw):
 @pytest.mark.parametrize("kw,code", [
     (dict(head_dim=64), -3), (dict(block_tokens=8), -3), (dict(n_kv_heads=3, n_q_heads=3), -3),
     (dict(n_q_heads=36), -3), (dict(pool_slots=32), -4), (dict(budget_blocks=4), -1),
-    (dict(max_blocks=1 << 20), -3), (dict(max_batch=0), -1), (dict(wait_limit_us=-5), -1), (dict(test_hold_producer=7), -1)])
+    (dict(max_blocks=1 << 20), -3), (dict(max_batch=0), -1), (dict(wait_limit_us=-5), -1), (dict(test_hold_producer=7), -1), (dict(attn_mode=3), -1)])
 def test_create_rejects_bad_configs_before_touching_the_device(kw, code):
     lib = pkg.load_library()
     cfg, _keep = _cfg(**kw)
