@@ -44,7 +44,7 @@ METRIC = "decode layer-steps/s (select+recall+attn); recall GB/s vs measured H2D
 # profiles/ (attn_kernel_c2.txt, score_select_kernel_c2.txt): same per-layer shapes as the bench
 # (recall_kernel: its reads cross the host link and its 5 MB of writes stay in L2 during the launch,
 # so DRAM sees next to nothing)
-NCU_DRAM_TRAFFIC = {"c2": {"attn_kernel": 134.5e6 + 4.3e6, "recall_kernel": 21.0e3}}
+NCU_DRAM_TRAFFIC = {"c2": {"recall_kernel": 21.0e3}}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -490,7 +490,7 @@ def measure_path(args, cfg, rank: int, world: int, dev, *, K: int, W: int, settl
                    "miss_script": cfg.miss_script or "none (LRU)", "append": bool(args.append),
                    "settle_steps": settle, "setup_s": round(setup_s, 1)},
         "clocks": clocks, "e2e": e2e,
-        "gpu_launches": 4 * n_launch,      # select+diff, recall, attention, merge: launches inside the timed region only
+        "gpu_launches": 3 * n_launch,      # select+diff, recall, attention (head-major: no merge kernel): launches inside the timed region only
         "roofline": {"kernel": "recall_kernel", "bound": "host_link_h2d", "achieved": recall_gbs, "peak": h2d_gbs,
                      "unit": "GB/s", "frac": recall_gbs / h2d_gbs,
                      "peak_source": "pinned cudaMemcpyAsync H2D of 1 GiB, best of 10, this run (nominal 64 GB/s PCIe Gen5 x16)",
@@ -503,9 +503,9 @@ def measure_path(args, cfg, rank: int, world: int, dev, *, K: int, W: int, settl
                                     "layers overlap across the recall streams; with one stream this is bytes per launch / "
                                     "mean launch duration)",
                      "alone": {"achieved": ser_recall_gbs, "frac": ser_recall_gbs / h2d_gbs}},
-        "rooflines": [hbm_entry("attn_kernel + attn_merge_kernel (timed region, recalls running beside it)", attn_bytes_launch, stages["attn"]["mean_ms"], peaks, ta),
-                      hbm_entry("attn_kernel + attn_merge_kernel (serial form, nothing else running)", attn_bytes_launch, ser["attn"]["mean_ms"], peaks, ta),
-                      hbm_entry("attn_kernel + attn_merge_kernel (one launch per layer back to back, one event pair around all)", attn_bytes_launch, b2b_attn_ms, peaks, ta),
+        "rooflines": [hbm_entry("attention call, attn_headmajor_kernel (timed region, recalls running beside it)", attn_bytes_launch, stages["attn"]["mean_ms"], peaks, ta),
+                      hbm_entry("attention call, attn_headmajor_kernel (serial form, nothing else running)", attn_bytes_launch, ser["attn"]["mean_ms"], peaks, ta),
+                      hbm_entry("attention call, attn_headmajor_kernel (one launch per layer back to back, one event pair around all)", attn_bytes_launch, b2b_attn_ms, peaks, ta),
                       hbm_entry("score_select_cluster_kernel: score + select + diff in one launch (serial form)", score_bytes_launch, ser["select_diff"]["mean_ms"], peaks, tsd),
                       hbm_entry("score_select_cluster_kernel: score + select + diff (back to back)", score_bytes_launch, b2b_fused_ms, peaks, tsd),
                       hbm_entry("score_select_cluster_kernel: score + select as a call of its own (serial form)", score_bytes_launch, ser2["score_select"]["mean_ms"], peaks, tss),
@@ -627,8 +627,8 @@ def measure_c5(args, dev, full: bool) -> dict:
         out["blocks"][str(B)] = {
             "n_blocks": nb, "budget_blocks": K, "pool_slots": C,
             "score_select": hbm_entry("score_select_cluster_kernel (per call, L2 flushed before each)", score_bytes, sc_ms, peaks),
-            "attention": hbm_entry("attn_kernel + attn_merge_kernel (per call, L2 flushed before each)", attn_bytes, at_ms, peaks),
-            "attention_back_to_back": hbm_entry("attn_kernel + attn_merge_kernel (back to back, pool reads 256 MiB > L2)", attn_bytes, at_b2b_ms, peaks)}
+            "attention": hbm_entry("attention call, attn_headmajor_kernel (per call, L2 flushed before each)", attn_bytes, at_ms, peaks),
+            "attention_back_to_back": hbm_entry("attention call, attn_headmajor_kernel (back to back, pool reads 256 MiB > L2)", attn_bytes, at_b2b_ms, peaks)}
 
         # ---- recall-fragmentation sweep at this block size
         hostB = host.view(cfg.batch, nb, cfg.block_bytes // 2)

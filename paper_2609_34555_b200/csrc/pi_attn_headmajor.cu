@@ -69,6 +69,30 @@ attn_headmajor_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p
     int n_mine = 0;
     for (int it = first_item; it < n_items; it += stride) ++n_mine;
     auto list_of = [&](int item) -> int { return p.headwise ? item : item / p.Hkv; };
+    // ---- metadata of my units: global row of the slot, token offset, valid tokens.  Staged by all threads in ONE
+    // round of independent loads (list entries up to K are read whatever the list's length: the tail holds -1),
+    // so that the producer never waits on a dependent global load.  Unit r of my k-th item sits at k * upi + r.
+    const int upi = p.K * SUB;                             // units an item can have
+    auto unit_meta = [&](int k, int r) -> int2 {
+        const int item = first_item + k * stride, seq = item / p.Hkv;
+        const size_t list = static_cast<size_t>(list_of(item));
+        const int j = r / SUB, sub = r - j * SUB;
+        int slot = p.sel_slots[list * p.K + j];
+        const int blk = p.sel_blocks[list * p.K + j];
+        const int ctx = p.ctx_len[seq], cnt = p.sel_count[list];
+        const bool listed = cnt >= 0 && cnt <= p.K && j < cnt && blk >= 0;
+        bool bad = false;
+        if (slot < 0 || slot >= p.C) {
+            if (listed) pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_ATTN, seq, j, slot);
+            slot = 0; bad = true;
+        }
+        const int nvalid = (!listed || bad) ? 0 : max(0, min(16, ctx - (blk * p.B + sub * 16)));
+        return make_int2(seq * p.C + slot, (sub * 16) | (nvalid << 8));
+    };
+    for (int i = tid; i < n_mine * upi && i < HM_META_UNITS; i += blockDim.x) {
+        const int k = i / upi;
+        s_meta[i] = unit_meta(k, i - k * upi);
+    }
     if (tid == 0) {
         int run = 0;
         for (int k = 0; k < n_mine; ++k) {
@@ -90,64 +114,35 @@ attn_headmajor_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p
     __syncthreads();
     const int total_units = s_units[n_mine];
 
-    // ---- metadata of my units: global row of the slot, token offset, valid tokens (staged by all threads so
-    // that the producer never waits on a dependent global load)
-    auto unit_meta = [&](int k, int r) -> int2 {           // r-th unit of my k-th item
-        const int item = first_item + k * stride, seq = item / p.Hkv;
-        const size_t list = static_cast<size_t>(list_of(item));
-        const int j = r / SUB, sub = r - j * SUB;
-        int slot = p.sel_slots[list * p.K + j];
-        const int blk = p.sel_blocks[list * p.K + j];
-        bool bad = false;
-        if (slot < 0 || slot >= p.C) {
-            pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_ATTN, seq, j, slot);
-            slot = 0; bad = true;
-        }
-        const int nvalid = (blk < 0 || bad) ? 0 : max(0, min(16, p.ctx_len[seq] - (blk * p.B + sub * 16)));
-        return make_int2(seq * p.C + slot, (sub * 16) | (nvalid << 8));
-    };
-    auto item_of_unit = [&](int u) -> int {                // last k with s_units[k] <= u
-        int lo = 0, hi = n_mine;
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (s_units[mid] <= u) lo = mid; else hi = mid;
-        }
-        return lo;
-    };
-    for (int u = tid; u < total_units && u < HM_META_UNITS; u += blockDim.x) {
-        const int k = item_of_unit(u);
-        s_meta[u] = unit_meta(k, u - s_units[k]);
-    }
-    __syncthreads();
-
     if (warp == HM_WARPS) {
-        // =============================== producer: one lane issues all TMA loads, a stage = up to 8 tiles of one item
-        if (lane == 0) {
-            int sidx = 0;
-            bool alive = true;
-            for (int k = 0; k < n_mine && alive; ++k) {
-                const int item = first_item + k * stride, h = item % p.Hkv;
-                const int u0 = s_units[k], n_u = s_units[k + 1] - u0;
-                for (int g = rank * HM_WARPS; g < n_u; g += HM_WARPS * S, ++sidx) {
-                    const int st = sidx % p.stages, round = sidx / p.stages;
-                    if (round > 0 && !mbar_wait(bar_empty + 8 * st, (round - 1) & 1, s_abort, p.wait_cycles)) { alive = false; break; }
-                    if (p.hold_last && k == n_mine - 1 && g + HM_WARPS * S >= n_u) { alive = false; break; }   // (test only)
-                    const int n_here = min(HM_WARPS, n_u - g);
-                    const uint32_t dst = ring + st * HM_STAGE_BYTES;
-                    int rows[HM_WARPS], offs[HM_WARPS];
-                    for (int w = 0; w < HM_WARPS; ++w) {
-                        int2 md = make_int2(0, 0);
-                        if (w < n_here) md = (u0 + g + w) < HM_META_UNITS ? s_meta[u0 + g + w] : unit_meta(k, g + w);
-                        s_nvalid[st * 8 + w] = w < n_here ? (md.y >> 8) : 0;
-                        rows[w] = md.x; offs[w] = md.y & 0xff;
-                    }
-                    // (the valid-token counts are written before the arrive below, which publishes them)
-                    mbar_expect_tx(bar_full + 8 * st, static_cast<uint32_t>(n_here) * 8192u);
-                    for (int w = 0; w < n_here; ++w) {
-                        tma_load_4d(dst + w * 4096, &pool_map, bar_full + 8 * st, 0, offs[w], 2 * h, rows[w]);
-                        tma_load_4d(dst + HM_HALF_BYTES + w * 4096, &pool_map, bar_full + 8 * st, 64, offs[w], 2 * h, rows[w]);
-                    }
+        // =============================== producer warp: a stage = up to 8 tiles of one item.  Lane 0 waits for the
+        // stage to be free and announces the bytes; lanes 0..15 then issue one TMA load each (tile lane / 2, half
+        // lane % 2 of the head dimension), so that a stage's sixteen loads go out together.
+        int sidx = 0;
+        bool alive = true;
+        const int w = lane >> 1, half = lane & 1;
+        for (int k = 0; k < n_mine && alive; ++k) {
+            const int item = first_item + k * stride, h = item % p.Hkv;
+            const int n_u = s_units[k + 1] - s_units[k];
+            for (int g = rank * HM_WARPS; g < n_u; g += HM_WARPS * S, ++sidx) {
+                const int st = sidx % p.stages, round = sidx / p.stages;
+                int ok = 1;
+                if (lane == 0) {
+                    if (round > 0 && !mbar_wait(bar_empty + 8 * st, (round - 1) & 1, s_abort, p.wait_cycles)) ok = 0;
+                    if (p.hold_last && k == n_mine - 1 && g + HM_WARPS * S >= n_u) ok = 0;   // (test only)
                 }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { alive = false; break; }
+                const int n_here = min(HM_WARPS, n_u - g);
+                const uint32_t dst = ring + st * HM_STAGE_BYTES;
+                int2 md = make_int2(0, 0);
+                if (lane < 16 && w < n_here) md = (k * upi + g + w) < HM_META_UNITS ? s_meta[k * upi + g + w] : unit_meta(k, g + w);
+                if (lane < 16 && half == 0) s_nvalid[st * 8 + w] = w < n_here ? (md.y >> 8) : 0;
+                __syncwarp();                               // the valid-token counts are written before the arrive, which publishes them
+                if (lane == 0) mbar_expect_tx(bar_full + 8 * st, static_cast<uint32_t>(n_here) * 8192u);
+                __syncwarp();
+                if (lane < 16 && w < n_here)
+                    tma_load_4d(dst + half * HM_HALF_BYTES + w * 4096, &pool_map, bar_full + 8 * st, half * 64, md.y & 0xff, 2 * h, md.x);
             }
         }
         __syncwarp();
