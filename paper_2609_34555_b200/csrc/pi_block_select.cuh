@@ -257,7 +257,9 @@ __device__ __forceinline__ unsigned block_topk_emit(const uint32_t* keys, int n,
     const unsigned t = histogram_walk<NT, AGGREGATE>(keys, m_lo, m_hi, sc, bn, k, above, cnt);
     unsigned need = k - above;                        // winners still to come from bucket t
 
-    if (cnt > RESOLVE_MAX || (!bn.linear && (bn.shift == 0 || cnt == need))) {
+    const Share sh = share_of<NT>(n);
+    const bool wide = (n + NT - 1) / NT > 64;         // more keys per thread than the winner masks below hold
+    if (cnt > RESOLVE_MAX || wide || (!bn.linear && (bn.shift == 0 || cnt == need))) {
         // Thresholds instead of a gathered bucket: one key value per bin, a bucket that wins as a whole,
         // or a crowded bucket (many equal or nearly equal keys) that further passes over the key bits narrow.
         uint32_t lo, hi;
@@ -284,18 +286,26 @@ __device__ __forceinline__ unsigned block_topk_emit(const uint32_t* keys, int n,
         return block_emit_ordered<NT, OUTSIDE_TAKEN>(keys, n, m_lo, m_hi, r, sc, emit);
     }
 
-    // ---- the bucket's keys are gathered while the sure winners (higher bins) are counted
-    const Share sh = share_of<NT>(n);
+    // ---- the bucket's keys are gathered while the sure winners (higher bins) are counted; every thread
+    // remembers which of its keys are sure winners and which sit in the bucket (bit j = its j-th key), so
+    // that the emission below touches the winners only
+    unsigned long long sure_mask = 0ull, bucket_mask = 0ull;
     unsigned c_sure = 0;
 #pragma unroll 4
     for (int i = sh.i0; i < sh.i1; ++i) {
-        if (i < m_lo || i >= m_hi) { c_sure += OUTSIDE_TAKEN ? 1u : 0u; continue; }
+        const unsigned long long bit = 1ull << (i - sh.i0);
+        if (i < m_lo || i >= m_hi) {
+            if (OUTSIDE_TAKEN) { sure_mask |= bit; ++c_sure; }
+            continue;
+        }
         const uint32_t key = keys[padded(i)];
         const unsigned b = bn.bin(key);
         if (b == t) {
             const unsigned p = atomicAdd(&sc.ncand, 1u);
             if (p < RESOLVE_MAX) { sc.cand_key[p] = key; sc.cand_idx[p] = i; }
+            bucket_mask |= bit;
         } else if (b != 0xffffffffu && b > t) {
+            sure_mask |= bit;
             ++c_sure;
         }
     }
@@ -315,23 +325,19 @@ __device__ __forceinline__ unsigned block_topk_emit(const uint32_t* keys, int n,
         const int oi = __shfl_sync(0xffffffffu, mi, j);
         pos += (((winmask >> j) & 1u) && oi < sh.i0) ? 1u : 0u;
     }
-#pragma unroll 4
-    for (int i = sh.i0; i < sh.i1; ++i) {
-        bool take;
-        uint32_t key = 0;
-        if (i < m_lo || i >= m_hi) take = OUTSIDE_TAKEN;
-        else {
-            key = keys[padded(i)];
-            const unsigned b = bn.bin(key);
-            if (b == t) {                             // a bucket key: did its candidate make it?
-                take = false;
-                for (unsigned c = 0; c < cnt; ++c)
-                    if (sc.cand_idx[c] == i) take = (winmask >> c) & 1u;
-            } else {
-                take = b != 0xffffffffu && b > t;
-            }
-        }
-        if (take) { emit(pos, i, key); ++pos; }
+    // my bucket keys whose candidate made it join my sure winners
+    while (bucket_mask) {
+        const int j = __ffsll(static_cast<long long>(bucket_mask)) - 1;
+        bucket_mask &= bucket_mask - 1;
+        for (unsigned c = 0; c < cnt; ++c)
+            if (sc.cand_idx[c] == sh.i0 + j && ((winmask >> c) & 1u)) sure_mask |= 1ull << j;
+    }
+    while (sure_mask) {
+        const int j = __ffsll(static_cast<long long>(sure_mask)) - 1;
+        sure_mask &= sure_mask - 1;
+        const int i = sh.i0 + j;
+        emit(pos, i, (i < m_lo || i >= m_hi) ? 0u : keys[padded(i)]);
+        ++pos;
     }
     return total_sure + static_cast<unsigned>(__popc(winmask));
 }

@@ -111,6 +111,22 @@ score_select_cluster_kernel(SDParams p) {
     }
     if (rank == 0) {
         pi_select::clear<SD_THREADS>(sc);
+        // The rows this CTA writes at the very end are touched now: the address translation of a page an SM has
+        // not used yet takes a microsecond or two, and at the end of the launch nothing would hide it.
+        if (tid < 8) {
+            const void* row = nullptr;
+            switch (tid) {
+                case 0: row = p.sel + static_cast<size_t>(seq) * p.K; break;
+                case 1: row = p.sel_count + seq; break;
+                case 2: row = FUSED ? static_cast<const void*>(p.sel_slots + static_cast<size_t>(seq) * p.K) : nullptr; break;
+                case 3: row = FUSED ? static_cast<const void*>(p.list + static_cast<size_t>(seq) * p.K) : nullptr; break;
+                case 4: row = FUSED ? static_cast<const void*>(p.count + seq) : nullptr; break;
+                case 5: row = FUSED ? static_cast<const void*>(p.stats) : nullptr; break;
+                case 6: row = p.scores ? static_cast<const void*>(p.scores + static_cast<size_t>(seq) * p.max_blocks) : nullptr; break;
+                default: row = FUSED ? static_cast<const void*>(p.step_dev) : nullptr; break;
+            }
+            if (row) asm volatile("prefetch.global.L2 [%0];" ::"l"(row));
+        }
         if (FUSED) {
             // what the diff needs besides the selection, fetched while the digests stream in
             const int32_t* sb = p.slot_block + static_cast<size_t>(seq) * p.C;
