@@ -54,7 +54,8 @@ struct Smem {
 // Bytes of the arrays above (without the key union), and of the union.
 __host__ __device__ inline size_t smem_lists_bytes(int K, int C) {
     const size_t kv = static_cast<size_t>(K < RANK_MAX_MISSES ? K : RANK_MAX_MISSES);
-    return (3 * static_cast<size_t>(K) + 3 * kv + 2 * static_cast<size_t>(C)) * 4 + ((static_cast<size_t>(C) + 15) & ~size_t(15));
+    const size_t words = (3 * static_cast<size_t>(K) + 3 * kv + 2 * static_cast<size_t>(C)) * 4;
+    return ((words + 15) & ~size_t(15)) + ((static_cast<size_t>(C) + 15) & ~size_t(15));
 }
 __host__ __device__ inline size_t smem_keys_bytes(int C, int Cpad) {
     const size_t a = (static_cast<size_t>(C) + C / 32 + 1) * 4, b = static_cast<size_t>(Cpad) * 8;

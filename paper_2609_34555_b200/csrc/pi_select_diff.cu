@@ -82,6 +82,9 @@ __device__ __forceinline__ void st_shared_cluster(uint32_t addr, uint32_t v) {
 __device__ __forceinline__ void cp_async4(void* smem, const void* gmem) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem))), "l"(gmem) : "memory");
 }
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem))), "l"(gmem) : "memory");
+}
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 template <bool FUSED>
@@ -109,41 +112,6 @@ score_select_cluster_kernel(SDParams p) {
         m = pi_diff::carve(smem_raw + p.key_bytes, p.K, p.C);
         s_table = reinterpret_cast<int32_t*>(smem_raw + p.key_bytes + pi_diff::smem_lists_bytes(p.K, p.C));
     }
-    if (rank == 0) {
-        pi_select::clear<SD_THREADS>(sc);
-        // The rows this CTA writes at the very end are touched now: the address translation of a page an SM has
-        // not used yet takes a microsecond or two, and at the end of the launch nothing would hide it.
-        if (tid < 8) {
-            const void* row = nullptr;
-            switch (tid) {
-                case 0: row = p.sel + static_cast<size_t>(seq) * p.K; break;
-                case 1: row = p.sel_count + seq; break;
-                case 2: row = FUSED ? static_cast<const void*>(p.sel_slots + static_cast<size_t>(seq) * p.K) : nullptr; break;
-                case 3: row = FUSED ? static_cast<const void*>(p.list + static_cast<size_t>(seq) * p.K) : nullptr; break;
-                case 4: row = FUSED ? static_cast<const void*>(p.count + seq) : nullptr; break;
-                case 5: row = FUSED ? static_cast<const void*>(p.stats) : nullptr; break;
-                case 6: row = p.scores ? static_cast<const void*>(p.scores + static_cast<size_t>(seq) * p.max_blocks) : nullptr; break;
-                default: row = FUSED ? static_cast<const void*>(p.step_dev) : nullptr; break;
-            }
-            if (row) asm volatile("prefetch.global.L2 [%0];" ::"l"(row));
-        }
-        if (FUSED) {
-            // what the diff needs besides the selection, fetched while the digests stream in
-            const int32_t* sb = p.slot_block + static_cast<size_t>(seq) * p.C;
-            const uint32_t* stp = p.slot_stamp + static_cast<size_t>(seq) * p.C;
-            for (int s = tid; s < p.C; s += SD_THREADS) {
-                cp_async4(m.sb + s, sb + s);
-                cp_async4(m.stp + s, stp + s);
-                m.used[s] = 0;
-            }
-            if (p.table_in_smem) {
-                const int32_t* row = p.table + static_cast<size_t>(seq) * p.max_blocks;
-                for (int b = tid; b < p.max_blocks; b += SD_THREADS) cp_async4(s_table + b, row + b);
-            }
-            if (tid == 0) s_ncand = 0;
-        }
-    }
-
     // ---------------- scoring: this CTA's share of the sequence, two chunks (16 loads per lane) a round
     const int blk_lo = static_cast<int>(rank) * p.cpc * SD_CHUNK;
     const uint4* dg = p.digest + static_cast<size_t>(seq) * p.max_blocks * 32;        // 32 uint4 per block
@@ -178,6 +146,46 @@ score_select_cluster_kernel(SDParams p) {
     };
     issue(va, 0);
     if (SD_TWO_SETS) issue(vb, 1);
+    // The first loads of the digests are in flight; what else the launch needs is set up behind them.
+    if (rank == 0) {
+        pi_select::clear<SD_THREADS>(sc);
+        // The rows this CTA writes at the very end are touched now: the address translation of a page an SM has
+        // not used yet takes a microsecond or two, and at the end of the launch nothing would hide it.
+        if (tid < 8) {
+            const void* row = nullptr;
+            switch (tid) {
+                case 0: row = p.sel + static_cast<size_t>(seq) * p.K; break;
+                case 1: row = p.sel_count + seq; break;
+                case 2: row = FUSED ? static_cast<const void*>(p.sel_slots + static_cast<size_t>(seq) * p.K) : nullptr; break;
+                case 3: row = FUSED ? static_cast<const void*>(p.list + static_cast<size_t>(seq) * p.K) : nullptr; break;
+                case 4: row = FUSED ? static_cast<const void*>(p.count + seq) : nullptr; break;
+                case 5: row = FUSED ? static_cast<const void*>(p.stats) : nullptr; break;
+                case 6: row = p.scores ? static_cast<const void*>(p.scores + static_cast<size_t>(seq) * p.max_blocks) : nullptr; break;
+                default: row = FUSED ? static_cast<const void*>(p.step_dev) : nullptr; break;
+            }
+            if (row) asm volatile("prefetch.global.L2 [%0];" ::"l"(row));
+        }
+        if (FUSED) {
+            // what the diff needs besides the selection, fetched while the digests stream in
+            const int32_t* sb = p.slot_block + static_cast<size_t>(seq) * p.C;
+            const uint32_t* stp = p.slot_stamp + static_cast<size_t>(seq) * p.C;
+            for (int s = tid; s < p.C; s += SD_THREADS) {
+                cp_async4(m.sb + s, sb + s);
+                cp_async4(m.stp + s, stp + s);
+                m.used[s] = 0;
+            }
+            if (p.table_in_smem) {
+                const int32_t* row = p.table + static_cast<size_t>(seq) * p.max_blocks;
+                if (((reinterpret_cast<uintptr_t>(row) | reinterpret_cast<uintptr_t>(s_table)) & 15) == 0 && (p.max_blocks & 3) == 0) {
+                    for (int b = tid * 4; b < p.max_blocks; b += SD_THREADS * 4) cp_async16(s_table + b, row + b);
+                } else {
+                    for (int b = tid; b < p.max_blocks; b += SD_THREADS) cp_async4(s_table + b, row + b);
+                }
+            }
+            if (tid == 0) s_ncand = 0;
+        }
+    }
+
     {
         pi_score::load_q_weights(p.q + (static_cast<size_t>(seq) * p.Hq + static_cast<size_t>(p.h_star) * p.G) * PI_HEAD_DIM,
                                  p.G, lane, w);
