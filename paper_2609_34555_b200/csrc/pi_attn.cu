@@ -258,6 +258,7 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
     if (warp == p.Hkv) {
         // =============================== producer: one lane issues all TMA loads
         if (lane == 0) {
+            const unsigned long long stream_policy = pi_l2_stream_policy();
             int seq = seq_of_unit(s_pref, p.batch, u0);
             for (int u = u0, it = 0; u < u1; ++u, ++it) {
                 while (u >= s_pref[seq + 1]) ++seq;
@@ -275,15 +276,15 @@ attn_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p) {
                     }
                     mbar_expect_tx(bar_full + 8 * st, stage_bytes);
                     for (int hh = 0; hh < p.Hkv; ++hh) {
-                        tma_load_4d(dst + hh * 4096, &pool_map, bar_full + 8 * st, 0, offs[hh], 2 * hh, rows[hh]);
-                        tma_load_4d(dst + half_bytes + hh * 4096, &pool_map, bar_full + 8 * st, 64, offs[hh], 2 * hh, rows[hh]);
+                        tma_load_4d(dst + hh * 4096, &pool_map, bar_full + 8 * st, 0, offs[hh], 2 * hh, rows[hh], stream_policy);
+                        tma_load_4d(dst + half_bytes + hh * 4096, &pool_map, bar_full + 8 * st, 64, offs[hh], 2 * hh, rows[hh], stream_policy);
                     }
                 } else {
                     const int2 md = it < meta_units ? s_meta[it] : unit_meta(u, seq, 0);
                     s_nvalid[st * 8] = md.y >> 8;
                     mbar_expect_tx(bar_full + 8 * st, stage_bytes);
-                    tma_load_4d(dst, &pool_map, bar_full + 8 * st, 0, md.y & 0xff, 0, md.x);
-                    tma_load_4d(dst + half_bytes, &pool_map, bar_full + 8 * st, 64, md.y & 0xff, 0, md.x);
+                    tma_load_4d(dst, &pool_map, bar_full + 8 * st, 0, md.y & 0xff, 0, md.x, stream_policy);
+                    tma_load_4d(dst + half_bytes, &pool_map, bar_full + 8 * st, 64, md.y & 0xff, 0, md.x, stream_policy);
                 }
             }
         }

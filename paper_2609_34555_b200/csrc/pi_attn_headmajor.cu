@@ -121,6 +121,7 @@ attn_headmajor_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p
         int sidx = 0;
         bool alive = true;
         const int w = lane >> 1, half = lane & 1;
+        const unsigned long long stream_policy = pi_l2_stream_policy();
         for (int k = 0; k < n_mine && alive; ++k) {
             const int item = first_item + k * stride, h = item % p.Hkv;
             const int n_u = s_units[k + 1] - s_units[k];
@@ -142,7 +143,7 @@ attn_headmajor_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p
                 if (lane == 0) mbar_expect_tx(bar_full + 8 * st, static_cast<uint32_t>(n_here) * 8192u);
                 __syncwarp();
                 if (lane < 16 && w < n_here)
-                    tma_load_4d(dst + half * HM_HALF_BYTES + w * 4096, &pool_map, bar_full + 8 * st, half * 64, md.y & 0xff, 2 * h, md.x);
+                    tma_load_4d(dst + half * HM_HALF_BYTES + w * 4096, &pool_map, bar_full + 8 * st, half * 64, md.y & 0xff, 2 * h, md.x, stream_policy);
             }
         }
         __syncwarp();

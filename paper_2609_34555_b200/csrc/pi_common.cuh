@@ -26,6 +26,20 @@
 __device__ __forceinline__ void pi_grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pi_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// L2 policy for data that is read once per layer-step (digests, pool blocks): its lines are the first to
+// go.  A layer-step streams more bytes than L2 holds; without the hint that stream pushes out what every
+// launch needs again -- tables, lists, queries and the kernels' own code, whose refetch from HBM costs the
+// serial tail of a launch several microseconds.
+__device__ __forceinline__ unsigned long long pi_l2_stream_policy() {
+    unsigned long long pol;
+#ifdef PI_NO_L2_HINTS
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+#else
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+#endif
+    return pol;
+}
+
 template <typename... KArgs, typename... Args>
 inline cudaError_t pi_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
                                  Args&&... args) {

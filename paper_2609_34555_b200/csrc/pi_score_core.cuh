@@ -28,6 +28,13 @@ __device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
     return v;
 }
 
+__device__ __forceinline__ uint4 ld_stream16(const uint4* p, unsigned long long policy) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(policy));
+    return v;
+}
+
 __device__ __forceinline__ float dot8(uint4 v, const float (&w)[8]) {
     float2 a = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&v.x));
     float2 b = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&v.y));

@@ -273,10 +273,11 @@ score_select_kernel(SelParams p) {
             const uint4* dg = p.digest + (static_cast<size_t>(rseq) * p.max_blocks * dig_heads +
                                           (dig_heads > 1 ? head : 0)) * 32;            // 32 uint4 per (block, head)
             uint4 v[BLOCKS_PER_WARP];
+            const unsigned long long stream_policy = pi_l2_stream_policy();
 #pragma unroll
             for (int i = 0; i < BLOCKS_PER_WARP; ++i) {
                 v[i] = make_uint4(0, 0, 0, 0);
-                if (b0 + i < p.max_blocks) v[i] = ld_stream16(dg + static_cast<size_t>(b0 + i) * dig_heads * 32 + lane);
+                if (b0 + i < p.max_blocks) v[i] = ld_stream16(dg + static_cast<size_t>(b0 + i) * dig_heads * 32 + lane, stream_policy);
             }
             if (c == f || n_sum > 1) {
                 pi_score::load_q_weights(p.q + (static_cast<size_t>(rseq) * p.Hq + static_cast<size_t>(head) * p.G) * PI_HEAD_DIM,

@@ -123,12 +123,13 @@ score_select_cluster_kernel(SDParams p) {
     // next are already in flight (8 to 16 independent 16-byte loads per lane at any time).  Digest rows up
     // to max_blocks are allocated, so they are read whatever the sequence's length and masked afterwards.
     uint4 va[BLOCKS_PER_WARP], vb[BLOCKS_PER_WARP];
+    const unsigned long long stream_policy = pi_l2_stream_policy();
     auto issue = [&](uint4 (&v)[BLOCKS_PER_WARP], int c) {
         const int b0 = blk_lo + c * SD_CHUNK + warp * BLOCKS_PER_WARP;
 #pragma unroll
         for (int i = 0; i < BLOCKS_PER_WARP; ++i) {
             v[i] = make_uint4(0, 0, 0, 0);
-            if (c < p.cpc && b0 + i < p.max_blocks) v[i] = pi_score::ld_stream16(dg + static_cast<size_t>(b0 + i) * 32 + lane);
+            if (c < p.cpc && b0 + i < p.max_blocks) v[i] = pi_score::ld_stream16(dg + static_cast<size_t>(b0 + i) * 32 + lane, stream_policy);
         }
     };
     auto finish = [&](uint4 (&v)[BLOCKS_PER_WARP], int c) {
