@@ -238,7 +238,7 @@ def measure_path(args, cfg, rank: int, world: int, dev, *, K: int, W: int, settl
     n_serial = min(K, 4)
     n_graph = min(K, 16) if "graph" in legs else 0
     n_hist = n_serial if "hist" in legs else 0
-    total_steps = settle + W + K + 6 * n_serial + n_e2e + n_graph + 4
+    total_steps = settle + W + K + 8 * n_serial + n_e2e + n_graph + 4
     pi, sess, R = build_session(cfg, rank, host_layers, world, args.recall_ctas,
                                 ctx_start=cfg.ctx - total_steps - 1 if args.append else 0, paged=args.paged,
                                 recall_streams=args.recall_streams, attn_ctas=args.attn_ctas)
@@ -353,6 +353,12 @@ def measure_path(args, cfg, rank: int, world: int, dev, *, K: int, W: int, settl
     serial2_ms, ser2, _ = serial_leg(True)
     serial2_plain_ms, _, _ = serial_leg(False)
     sess.fused_select_diff = True
+    # and with the attention split around the recall: the recall on a stream of its own, the resident blocks'
+    # share of the attention beside it, the recalled blocks' share once it has landed
+    sess.split_attention = True
+    serial3_ms, ser3, _ = serial_leg(True)
+    serial3_plain_ms, _, _ = serial_leg(False)
+    sess.split_attention = False
 
     # ---------------- distribution of the miss counts: a few more steps, read back after each
     # (per sequence and layer-step: units of the recall lists)
@@ -519,6 +525,11 @@ def measure_path(args, cfg, rank: int, world: int, dev, *, K: int, W: int, settl
         "serial": {"layer_steps_per_s": cfg.n_layers / (serial_ms * 1e-3),
                    "layer_steps_per_s_without_events": cfg.n_layers / (serial_plain_ms * 1e-3),
                    "stages_us": {k: v["mean_ms"] * 1e3 for k, v in ser.items() if v["launches"]},
+                   "attention_split_around_the_recall": {
+                       "layer_steps_per_s": cfg.n_layers / (serial3_ms * 1e-3),
+                       "layer_steps_per_s_without_events": cfg.n_layers / (serial3_plain_ms * 1e-3),
+                       "stages_us": {k: v["mean_ms"] * 1e3 for k, v in ser3.items() if v["launches"]},
+                       "note": "pi_sparse_decode_attn_resident runs beside the recall, pi_sparse_decode_attn_recalled ('attn') after it"},
                    "selection_and_diff_as_two_calls": {
                        "layer_steps_per_s": cfg.n_layers / (serial2_ms * 1e-3),
                        "layer_steps_per_s_without_events": cfg.n_layers / (serial2_plain_ms * 1e-3),

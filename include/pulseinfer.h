@@ -225,6 +225,39 @@ int pi_sparse_decode_attn(pi_ctx* ctx, int layer, int batch, const void* q_dev, 
                           const int32_t* sel_count_dev, const int32_t* ctx_len_dev, void* out_dev,
                           float* lse_dev, void* stream);
 
+/* The same attention split around the recall (Sec. 4.2.1: the recall of the missing blocks and the
+ * attention are two stages of a layer; the selected blocks that were already resident do not wait for
+ * the first).  The miss diff never evicts a block of the current selection, so
+ *   pi_sparse_decode_attn_resident  may run as soon as pi_diff_misses (or pi_score_select_diff) has
+ *       finished, beside pi_recall_gather_scatter: it covers the selected blocks whose slot is not a
+ *       destination of recall_list_dev and leaves its softmax state in state_dev;
+ *   pi_sparse_decode_attn_recalled  runs after both: it covers the blocks the recall brought in,
+ *       folds the state in and writes out_dev.
+ * Together they compute what pi_sparse_decode_attn computes (same arithmetic per block, the two
+ * partial softmax states merged once more; results agree to fp32 rounding, not bit for bit).
+ *   recall_list_dev / list_capacity / recall_count_dev: this step's lists of the shared selection as
+ *       pi_diff_misses wrote them (one list per sequence, units = blocks, dst_unit = pool slot)
+ *   state_dev: device scratch of pi_attn_state_bytes(ctx, batch) bytes, 16-byte aligned, owned by the
+ *       caller; written by the first call, read by the second; contents are private to the library
+ *   the other arguments: as pi_sparse_decode_attn (no lse output).
+ * Ordering is the caller's: _resident after the diff, _recalled after _resident and after the recall.
+ * Shapes the split form does not cover (the attention runs in its flat form, or a CTA's blocks exceed
+ * the staged metadata): _resident returns PI_OK without launching anything and _recalled computes the
+ * whole attention, so the pair can be called unconditionally. */
+int pi_sparse_decode_attn_resident(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* pool_dev,
+                                   const int32_t* sel_slots_dev, const int32_t* sel_blocks_dev,
+                                   const int32_t* sel_count_dev, const int32_t* ctx_len_dev,
+                                   const pi_extent* recall_list_dev, int32_t list_capacity,
+                                   const int32_t* recall_count_dev, float* state_dev, void* stream);
+int pi_sparse_decode_attn_recalled(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* pool_dev,
+                                   const int32_t* sel_slots_dev, const int32_t* sel_blocks_dev,
+                                   const int32_t* sel_count_dev, const int32_t* ctx_len_dev,
+                                   const pi_extent* recall_list_dev, int32_t list_capacity,
+                                   const int32_t* recall_count_dev, const float* state_dev, void* out_dev,
+                                   void* stream);
+/* Bytes of state_dev for `batch` sequences (> 0), or a negative PI_ERR_* code. */
+int64_t pi_attn_state_bytes(pi_ctx* ctx, int batch);
+
 /* The same attention when every KV head carries its own selection (the headwise strategy of the
  * paper's selection study, Sec. 4.4.1, as produced by pi_score_select_strategy(PI_SELECT_HEADWISE) +
  * pi_diff_misses over batch*Hkv rows + per-head fragment recall): query heads of KV head h attend

@@ -23,7 +23,7 @@ ERR_NAMES = {
 EXTENT_DTYPE = torch.int32      # a pi_extent is four int32: src_unit, dst_unit, n_units, units_before
 
 EXPORTS = ["pi_create", "pi_destroy", "pi_score_select", "pi_score_select_diff", "pi_score_select_diff_devstep", "pi_score_select_noalloc", "pi_score_select_strategy", "pi_diff_misses", "pi_diff_misses_devstep", "pi_recall_gather_scatter",
-           "pi_recall_gather_scatter_paged", "pi_sparse_decode_attn", "pi_sparse_decode_attn_headwise", "pi_append_kv", "pi_append_kv_paged", "pi_append_kv_devstep", "pi_build_digests", "pi_build_digests_all", "pi_table_init", "pi_h2d_copy_ms", "pi_empty_launch", "pi_middle_attention_mass",
+           "pi_recall_gather_scatter_paged", "pi_sparse_decode_attn", "pi_sparse_decode_attn_headwise", "pi_sparse_decode_attn_resident", "pi_sparse_decode_attn_recalled", "pi_attn_state_bytes", "pi_append_kv", "pi_append_kv_paged", "pi_append_kv_devstep", "pi_build_digests", "pi_build_digests_all", "pi_table_init", "pi_h2d_copy_ms", "pi_empty_launch", "pi_middle_attention_mass",
            "pi_get_status", "pi_get_stats", "pi_clear_status", "pi_strerror"]
 
 
@@ -73,6 +73,9 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.pi_build_digests_all.argtypes = [c_void_p, c_int, vp, c_int64, i32p, vp, vp]
     lib.pi_sparse_decode_attn.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, i32p, vp, vp, vp]
     lib.pi_sparse_decode_attn_headwise.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, i32p, vp, vp, vp]
+    lib.pi_sparse_decode_attn_resident.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, i32p, vp, c_int32, i32p, vp, vp]
+    lib.pi_sparse_decode_attn_recalled.argtypes = [c_void_p, c_int, c_int, vp, vp, i32p, i32p, i32p, i32p, vp, c_int32, i32p, vp, vp, vp]
+    lib.pi_attn_state_bytes.argtypes = [c_void_p, c_int]
     lib.pi_append_kv.argtypes = [c_void_p, c_int, c_int, c_uint32, vp, vp, i32p, vp, c_int64, vp, i32p, i32p, u32p, vp, vp]
     lib.pi_build_digests.argtypes = [c_void_p, c_int, c_int, vp, c_int64, i32p, vp, vp]
     lib.pi_table_init.argtypes = [c_void_p, c_int, i32p, i32p, i32p, u32p, vp]
@@ -87,6 +90,7 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     for name in EXPORTS:
         if name != "pi_strerror":
             getattr(lib, name).restype = c_int
+    lib.pi_attn_state_bytes.restype = c_int64
     _lib = lib
     return lib
 
@@ -289,6 +293,42 @@ class PulseInfer:
             _dev(sel_count, torch.int32, "sel_count"), _dev(ctx_len, torch.int32, "ctx_len"),
             _dev(out, torch.bfloat16, "out"), None if lse is None else _dev(lse, torch.float32, "lse"),
             _stream(stream)))
+
+    def attn_state(self, batch: int, device=None) -> torch.Tensor:
+        """Scratch for the attention split around the recall (sparse_decode_attn_resident / _recalled)."""
+        n = self._lib.pi_attn_state_bytes(self._ctx, batch)
+        if n < 0:
+            raise PiError("pi_attn_state_bytes", int(n), strerror(int(n)))
+        return torch.empty(n // 4, dtype=torch.float32, device=device or torch.device("cuda"))
+
+    def sparse_decode_attn_resident(self, layer: int, q, pool, sel_slots, sel_blocks, sel_count, ctx_len, recall_list,
+                                    recall_count, state, stream=None) -> None:
+        """First half of the attention split around the recall: the selected blocks the step's recall list
+        does not touch; may run beside recall_gather_scatter.  Leaves its softmax state in `state`."""
+        batch = q.shape[0]
+        if not pool.is_cuda or not pool.is_contiguous():
+            raise TypeError("pool: expected a contiguous CUDA tensor")
+        _check("pi_sparse_decode_attn_resident", self._lib.pi_sparse_decode_attn_resident(
+            self._ctx, layer, batch, _dev(q, torch.bfloat16, "q"), pool.data_ptr(),
+            _dev(sel_slots, torch.int32, "sel_slots"), _dev(sel_blocks, torch.int32, "sel_blocks"),
+            _dev(sel_count, torch.int32, "sel_count"), _dev(ctx_len, torch.int32, "ctx_len"),
+            _dev(recall_list, torch.int32, "recall_list"), recall_list.shape[-2],
+            _dev(recall_count, torch.int32, "recall_count"), _dev(state, torch.float32, "state"), _stream(stream)))
+
+    def sparse_decode_attn_recalled(self, layer: int, q, pool, sel_slots, sel_blocks, sel_count, ctx_len, recall_list,
+                                    recall_count, state, out, stream=None) -> None:
+        """Second half: the blocks the recall brought in, merged with `state`; writes `out`.  The caller
+        orders it after the first half and after the recall."""
+        batch = q.shape[0]
+        if not pool.is_cuda or not pool.is_contiguous():
+            raise TypeError("pool: expected a contiguous CUDA tensor")
+        _check("pi_sparse_decode_attn_recalled", self._lib.pi_sparse_decode_attn_recalled(
+            self._ctx, layer, batch, _dev(q, torch.bfloat16, "q"), pool.data_ptr(),
+            _dev(sel_slots, torch.int32, "sel_slots"), _dev(sel_blocks, torch.int32, "sel_blocks"),
+            _dev(sel_count, torch.int32, "sel_count"), _dev(ctx_len, torch.int32, "ctx_len"),
+            _dev(recall_list, torch.int32, "recall_list"), recall_list.shape[-2],
+            _dev(recall_count, torch.int32, "recall_count"), _dev(state, torch.float32, "state"),
+            _dev(out, torch.bfloat16, "out"), _stream(stream)))
 
     def append_kv(self, layer: int, step: int, k_new, v_new, ctx_len, host_kv, pool, block_table, slot_block,
                   slot_stamp, digest, host_seq_stride: Optional[int] = None, page_table=None,

@@ -310,6 +310,56 @@ extern "C" int pi_sparse_decode_attn_headwise(pi_ctx* ctx, int layer, int batch,
                      out_dev, lse_dev, 1, stream);
 }
 
+// Attention split around the recall.  Where the head-major form with staged metadata does not apply the
+// first call does nothing and the second one is the whole attention.
+static int attn_phase_call(pi_ctx* ctx, int layer, int batch, int phase, const void* q_dev, const void* pool_dev,
+                           const int32_t* sel_slots_dev, const int32_t* sel_blocks_dev, const int32_t* sel_count_dev,
+                           const int32_t* ctx_len_dev, const pi_extent* recall_list_dev, int32_t list_capacity,
+                           const int32_t* recall_count_dev, float* state_dev, void* out_dev, void* stream) {
+    int rc = check_call(ctx, layer, batch);
+    if (rc != PI_OK) return rc;
+    if (!q_dev || !pool_dev || !sel_slots_dev || !sel_blocks_dev || !sel_count_dev || !ctx_len_dev ||
+        !recall_list_dev || !recall_count_dev || list_capacity < 1 || !state_dev || (phase == 2 && !out_dev))
+        return PI_ERR_INVALID_ARG;
+    if (!pi_aligned16(q_dev) || (out_dev && !pi_aligned16(out_dev)) || !pi_aligned16(state_dev) ||
+        !pi_aligned16(recall_list_dev) || (reinterpret_cast<uintptr_t>(pool_dev) & 127u))
+        return PI_ERR_BAD_ALIGN;
+    if (!pi_attn_phased_fits(ctx, batch)) {
+        if (phase == 1) return PI_OK;
+        return pi_launch_attn(ctx, batch, q_dev, pool_dev, sel_slots_dev, sel_blocks_dev, sel_count_dev, ctx_len_dev,
+                              out_dev, nullptr, 0, static_cast<cudaStream_t>(stream));
+    }
+    pi_attn_phase ph;
+    ph.phase = phase; ph.rlist = recall_list_dev; ph.rcap = list_capacity; ph.rcount = recall_count_dev; ph.state = state_dev;
+    return pi_launch_attn_headmajor(ctx, batch, q_dev, pool_dev, sel_slots_dev, sel_blocks_dev, sel_count_dev,
+                                    ctx_len_dev, out_dev, nullptr, 0, &ph, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int pi_sparse_decode_attn_resident(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* pool_dev,
+                                              const int32_t* sel_slots_dev, const int32_t* sel_blocks_dev,
+                                              const int32_t* sel_count_dev, const int32_t* ctx_len_dev,
+                                              const pi_extent* recall_list_dev, int32_t list_capacity,
+                                              const int32_t* recall_count_dev, float* state_dev, void* stream) {
+    return attn_phase_call(ctx, layer, batch, 1, q_dev, pool_dev, sel_slots_dev, sel_blocks_dev, sel_count_dev,
+                           ctx_len_dev, recall_list_dev, list_capacity, recall_count_dev, state_dev, nullptr, stream);
+}
+
+extern "C" int pi_sparse_decode_attn_recalled(pi_ctx* ctx, int layer, int batch, const void* q_dev, const void* pool_dev,
+                                              const int32_t* sel_slots_dev, const int32_t* sel_blocks_dev,
+                                              const int32_t* sel_count_dev, const int32_t* ctx_len_dev,
+                                              const pi_extent* recall_list_dev, int32_t list_capacity,
+                                              const int32_t* recall_count_dev, const float* state_dev, void* out_dev,
+                                              void* stream) {
+    return attn_phase_call(ctx, layer, batch, 2, q_dev, pool_dev, sel_slots_dev, sel_blocks_dev, sel_count_dev,
+                           ctx_len_dev, recall_list_dev, list_capacity, recall_count_dev, const_cast<float*>(state_dev),
+                           out_dev, stream);
+}
+
+extern "C" int64_t pi_attn_state_bytes(pi_ctx* ctx, int batch) {
+    if (!ctx || batch < 1 || batch > ctx->cfg.max_batch) return PI_ERR_INVALID_ARG;
+    return pi_attn_state_floats(ctx, batch) * 4;
+}
+
 static int append_call(pi_ctx* ctx, int layer, int batch, uint32_t step, const uint32_t* step_dev, const void* k_new_dev, const void* v_new_dev,
                        const int32_t* ctx_len_dev, void* host_kv_pinned, int64_t host_seq_stride_bytes,
                        const int32_t* page_table, int64_t page_stride, int32_t n_pages, void* pool_dev,

@@ -383,7 +383,7 @@ int pi_launch_attn(pi_ctx* c, int batch, const void* q, const void* pool, const 
     // the head-major form keeps everything inside the CTA (no partials, no merge kernel); it is taken when
     // (sequences x KV heads) fills the grid evenly, or when the configuration asks for it
     if (cfg.attn_mode == 2 || (cfg.attn_mode == 0 && pi_attn_headmajor_fits(c, batch, nullptr, nullptr, nullptr)))
-        return pi_launch_attn_headmajor(c, batch, q, pool, sel_slots, sel_blocks, sel_count, ctx_len, out, lse, headwise, stream);
+        return pi_launch_attn_headmajor(c, batch, q, pool, sel_slots, sel_blocks, sel_count, ctx_len, out, lse, headwise, nullptr, stream);
     const long long n_slots = static_cast<long long>(batch) * cfg.pool_slots;
     // the map is rebuilt when the pool, its size or the box (all heads / one head per load) changes
     if (c->pool_map_ptr != pool || c->pool_map_slots != n_slots || c->pool_map_headwise != headwise) {

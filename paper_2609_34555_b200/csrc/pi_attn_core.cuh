@@ -26,6 +26,12 @@ struct AttnParams {
     int hold_last;                // test only: the producer never issues the loads of its CTA's last unit
     long long wait_cycles;        // bound of every wait on a barrier
     float scale_log2;
+    // attention split around the recall (head-major form only): the step's recall list names the slots that are
+    // being filled; `state` carries the softmax state of the first call to the second
+    const pi_extent* rlist;
+    const int32_t* rcount;
+    int rcap;
+    float* state;                 // [items][NT * 36][32] fp32, a warp's state as the merge regions hold it
 };
 
 // Blocks of sequence s that the unit list walks: the selection's count, or, when every KV head has

@@ -14,6 +14,14 @@
 // cluster reads the others' final states out of their shared memory (distributed shared memory, plain
 // loads) and writes the result.  The same kernel serves per-head selections (the headwise strategy of
 // Sec. 4.4.1): item (s, h) then walks list (s, h).
+//
+// Split around the recall (PHASE 1 and 2): the blocks of a selection that were resident before the step do
+// not depend on the recall (the diff never evicts a selected block), so their share of the attention can run
+// while the missing blocks are still on their way.  PHASE 1 walks the selected blocks whose slot is not a
+// destination of the step's recall list and leaves the merged softmax state of every item in global memory;
+// PHASE 2 walks the others (a handful per sequence), folds that state in and writes the result.  Both build
+// the set of slots being filled from the recall list itself (a bitmap per item in shared memory) and compact
+// their units in selection order, so the split is a function of the lists alone.
 #include "pi_common.cuh"
 #include "pi_attn_core.cuh"
 
@@ -44,7 +52,7 @@ __device__ __forceinline__ uint32_t map_shared_rank(uint32_t addr, unsigned rank
     return r;
 }
 
-template <int NT>
+template <int NT, int PHASE>
 __global__ void __launch_bounds__(288, 1)
 attn_headmajor_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p, int n_items, int items_per_cta) {
     extern __shared__ unsigned char smem_dyn[];
@@ -57,6 +65,7 @@ attn_headmajor_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p
     int2* s_meta = reinterpret_cast<int2*>(s_abort + 2);                               // [HM_META_UNITS] {slot row, token offset | nvalid << 8}
     int* s_units = reinterpret_cast<int*>(s_meta + HM_META_UNITS);                     // [items_per_cta + 1] units before each of my items
     float* s_merge = reinterpret_cast<float*>(s_units + ((items_per_cta + 2 + 3) & ~3)); // [4][NT * 36][32]
+    unsigned* s_fresh = reinterpret_cast<unsigned*>(s_merge + 4 * NT * 36 * 32);         // PHASE: [items_per_cta][ceil(C / 32)] slots being filled
     const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + ATTN_MAX_STAGES);
     const int SUB = p.B >> 4;
     if (tid == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&pool_map) : "memory");
@@ -89,18 +98,73 @@ attn_headmajor_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p
         const int nvalid = (!listed || bad) ? 0 : max(0, min(16, ctx - (blk * p.B + sub * 16)));
         return make_int2(seq * p.C + slot, (sub * 16) | (nvalid << 8));
     };
-    for (int i = tid; i < n_mine * upi && i < HM_META_UNITS; i += blockDim.x) {
-        const int k = i / upi;
-        s_meta[i] = unit_meta(k, i - k * upi);
+    if (PHASE == 0) {
+        for (int i = tid; i < n_mine * upi && i < HM_META_UNITS; i += blockDim.x) {
+            const int k = i / upi;
+            s_meta[i] = unit_meta(k, i - k * upi);
+        }
+    } else {
+        // slots the step's recall fills, per item; then the kept units of every item, compacted in selection order
+        // (the launcher has checked that all of a CTA's units fit the staged metadata)
+        const int words = (p.C + 31) >> 5;
+        for (int i = tid; i < n_mine * words; i += blockDim.x) s_fresh[i] = 0u;
+        __syncthreads();
+        for (int k = 0; k < n_mine; ++k) {
+            const int seq = (first_item + k * stride) / p.Hkv;
+            int n = p.rcount[seq];
+            if (n < 0 || n > p.rcap) n = 0;                 // (the recall kernel reports such a count)
+            for (int e = tid; e < n; e += blockDim.x) {
+                const pi_extent x = p.rlist[static_cast<size_t>(seq) * p.rcap + e];
+                for (int u = 0; u < x.n_units; ++u) {
+                    const int slot = x.dst_unit + u;
+                    if (slot >= 0 && slot < p.C) atomicOr(&s_fresh[k * words + (slot >> 5)], 1u << (slot & 31));
+                }
+            }
+        }
+        __syncthreads();
+        for (int k = warp; k < n_mine; k += HM_WARPS + 1) {
+            const int item = first_item + k * stride, seq = item / p.Hkv;
+            int cnt = p.sel_count[seq];
+            if (cnt < 0 || cnt > p.K) cnt = 0;              // reported below
+            const int ctx = p.ctx_len[seq];
+            int kept = 0;
+            for (int base = 0; base < cnt; base += 32) {
+                const int j = base + lane;
+                bool keep = false;
+                int slot = 0, blk = -1;
+                if (j < cnt) {
+                    slot = p.sel_slots[static_cast<size_t>(seq) * p.K + j];
+                    blk = p.sel_blocks[static_cast<size_t>(seq) * p.K + j];
+                    if (slot < 0 || slot >= p.C) {
+                        if (blk >= 0 && PHASE == 1) pi_report(p.st, PI_ERR_INDEX_RANGE, PI_STAGE_ATTN, seq, j, slot);
+                    } else if (blk >= 0) {
+                        const bool fresh = (s_fresh[k * words + (slot >> 5)] >> (slot & 31)) & 1u;
+                        keep = fresh == (PHASE == 2);
+                    }
+                }
+                const unsigned b = __ballot_sync(0xffffffffu, keep);
+                if (keep) {
+                    const int pos = kept + __popc(b & ((1u << lane) - 1u));
+                    for (int sub = 0; sub < SUB; ++sub) {
+                        const int nvalid = max(0, min(16, ctx - (blk * p.B + sub * 16)));
+                        s_meta[k * upi + pos * SUB + sub] = make_int2(seq * p.C + slot, (sub * 16) | (nvalid << 8));
+                    }
+                }
+                kept += __popc(b);
+            }
+            if (lane == 0) s_units[k + 1] = kept * SUB;       // turned into a running sum below
+        }
+        __syncthreads();
     }
     if (tid == 0) {
         int run = 0;
         for (int k = 0; k < n_mine; ++k) {
             const int item = first_item + k * stride;
             int n = p.sel_count[list_of(item)];
-            if (n < 0 || n > p.K) { pi_report(p.st, PI_ERR_CAPACITY, PI_STAGE_ATTN, item / p.Hkv, n, p.K); n = 0; }
+            if (n < 0 || n > p.K) { if (PHASE != 2) pi_report(p.st, PI_ERR_CAPACITY, PI_STAGE_ATTN, item / p.Hkv, n, p.K); n = 0; }
+            const int units = PHASE == 0 ? n * SUB : s_units[k + 1];
             s_units[k] = run;
-            run += n * SUB;
+            run += units;
         }
         s_units[n_mine] = run;
         *s_abort = 0;
@@ -207,11 +271,24 @@ attn_headmajor_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p
             }
         attn_write_out<NT>(p, seq, h, row, colp, o, m, l);
     };
-    int last_seq = 0, last_h = 0;
+    // what an item ends with: the result (PHASE 0), its state left for the second call (PHASE 1), or the first
+    // call's state folded in before the result (PHASE 2).  Called by warp 0 of the CTA that holds the item's state.
+    auto conclude = [&](int item) {
+        if (PHASE == 1) {
+            put(p.state + static_cast<size_t>(item) * (NT * 36 * 32) + lane);
+            return;
+        }
+        if (PHASE == 2) {
+            const float* g = p.state + static_cast<size_t>(item) * (NT * 36 * 32) + lane;
+            take([&](int i) { return g[i * 32]; });
+        }
+        finish(item / p.Hkv, item % p.Hkv);
+    };
+    int last_item = 0;
     for (int k = 0; k < n_mine; ++k) {
         const int item = first_item + k * stride, seq = item / p.Hkv, h = item % p.Hkv;
         const int n_u = s_units[k + 1] - s_units[k];
-        last_seq = seq; last_h = h;
+        last_item = item;
         uint32_t bq[NT][8][2];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
@@ -255,7 +332,7 @@ attn_headmajor_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p
         if (warp == 0) {
             const float* r = region(0);
             take([&](int i) { return r[i * 32]; });
-            if (S == 1) finish(seq, h);
+            if (S == 1) conclude(item);
         }
     }
     if (S > 1) {
@@ -270,7 +347,7 @@ attn_headmajor_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p
                 const uint32_t theirs = map_shared_rank(mine, static_cast<unsigned>(r));
                 take([&](int i) { return ld_shared_cluster_f32(theirs + static_cast<uint32_t>(i) * 128u); });
             }
-            finish(last_seq, last_h);
+            conclude(last_item);
         }
         cluster_sync_all();                                 // nobody leaves while its state may still be read
     }
@@ -296,9 +373,31 @@ bool pi_attn_headmajor_fits(const pi_ctx* c, int batch, int* grid_out, int* item
     return grid * 5 >= ctas * 3 && static_cast<long long>(items) * split * 10 >= static_cast<long long>(rounds) * grid * 9;
 }
 
+static size_t hm_smem_bytes(const pi_config& cfg, int per_cta, int NT, int stages, bool phased) {
+    return 1024 + static_cast<size_t>(stages) * HM_STAGE_BYTES + 2 * ATTN_MAX_STAGES * 8 +
+           (ATTN_MAX_STAGES * 8 + 2) * 4 + HM_META_UNITS * 8 + ((static_cast<size_t>(per_cta) + 2 + 3) & ~size_t(3)) * 4 +
+           static_cast<size_t>(4) * NT * 36 * 32 * 4 + 16 +
+           (phased ? static_cast<size_t>(per_cta) * ((cfg.pool_slots + 31) / 32) * 4 : 0);
+}
+
+// The split around the recall needs the head-major form with every unit of a CTA in the staged metadata.
+bool pi_attn_phased_fits(const pi_ctx* c, int batch) {
+    int grid = 1, per_cta = 1, split = 1;
+    const bool fits = pi_attn_headmajor_fits(c, batch, &grid, &per_cta, &split);
+    if (c->cfg.attn_mode == 1 || (c->cfg.attn_mode == 0 && !fits)) return false;
+    if (c->cfg.n_kv_heads > 8) return false;
+    const long long units = static_cast<long long>(per_cta) * c->cfg.budget_blocks * (c->cfg.block_tokens / 16);
+    const int NT = c->cfg.n_q_heads / c->cfg.n_kv_heads <= 8 ? 1 : 2;
+    return units <= HM_META_UNITS && hm_smem_bytes(c->cfg, per_cta, NT, NT == 1 ? 3 : 2, true) <= 227 * 1024;
+}
+long long pi_attn_state_floats(const pi_ctx* c, int batch) {
+    const int NT = c->cfg.n_q_heads / c->cfg.n_kv_heads <= 8 ? 1 : 2;
+    return static_cast<long long>(batch) * c->cfg.n_kv_heads * NT * 36 * 32;
+}
+
 int pi_launch_attn_headmajor(pi_ctx* c, int batch, const void* q, const void* pool, const int32_t* sel_slots,
                              const int32_t* sel_blocks, const int32_t* sel_count, const int32_t* ctx_len, void* out,
-                             float* lse, int headwise, cudaStream_t stream) {
+                             float* lse, int headwise, const pi_attn_phase* phase, cudaStream_t stream) {
     const pi_config& cfg = c->cfg;
     const long long n_slots = static_cast<long long>(batch) * cfg.pool_slots;
     // the tensor map with a box of one head's K and V rows (shared with the headwise form of the flat kernel)
@@ -333,13 +432,16 @@ int pi_launch_attn_headmajor(pi_ctx* c, int batch, const void* q, const void* po
     p.hold_last = cfg.test_hold_producer;
     p.wait_cycles = c->wait_limit_cycles;
     p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(PI_HEAD_DIM));
+    const int ph = phase ? phase->phase : 0;
+    p.rlist = phase ? phase->rlist : nullptr;
+    p.rcount = phase ? phase->rcount : nullptr;
+    p.rcap = phase ? phase->rcap : 0;
+    p.state = phase ? phase->state : nullptr;
     const int NT = p.G <= 8 ? 1 : 2;
     p.stages = NT == 1 ? 3 : 2;                      // the wider merge regions of G > 8 take the room of a stage
     int grid = 1, per_cta = 1, split = 1;
     (void)pi_attn_headmajor_fits(c, batch, &grid, &per_cta, &split);
-    const size_t smem = 1024 + static_cast<size_t>(p.stages) * HM_STAGE_BYTES + 2 * ATTN_MAX_STAGES * 8 +
-                        (ATTN_MAX_STAGES * 8 + 2) * 4 + HM_META_UNITS * 8 + ((static_cast<size_t>(per_cta) + 2 + 3) & ~size_t(3)) * 4 +
-                        static_cast<size_t>(4) * NT * 36 * 32 * 4 + 16;
+    const size_t smem = hm_smem_bytes(cfg, per_cta, NT, p.stages, ph != 0);
     const int n_items = batch * cfg.n_kv_heads;
     auto launch = [&](auto kernel) -> int {
         PI_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
@@ -360,7 +462,10 @@ int pi_launch_attn_headmajor(pi_ctx* c, int batch, const void* q, const void* po
         PI_CUDA_TRY(cudaLaunchKernelEx(&lc, kernel, c->pool_map, p, n_items, per_cta));
         return PI_OK;
     };
-    const int rc = NT == 1 ? launch(attn_headmajor_kernel<1>) : launch(attn_headmajor_kernel<2>);
+    int rc;
+    if (ph == 0) rc = NT == 1 ? launch(attn_headmajor_kernel<1, 0>) : launch(attn_headmajor_kernel<2, 0>);
+    else if (ph == 1) rc = NT == 1 ? launch(attn_headmajor_kernel<1, 1>) : launch(attn_headmajor_kernel<2, 1>);
+    else rc = NT == 1 ? launch(attn_headmajor_kernel<1, 2>) : launch(attn_headmajor_kernel<2, 2>);
     if (rc != PI_OK) return rc;
     PI_CUDA_TRY(cudaGetLastError());
     return PI_OK;

@@ -143,9 +143,21 @@ int pi_launch_attn(pi_ctx*, int batch, const void* q, const void* pool, const in
                    void* out, float* lse, int headwise, cudaStream_t);
 // head-major form of the attention (one (sequence, KV head) per CTA); `fits` says whether the items fill the grid evenly
 bool pi_attn_headmajor_fits(const pi_ctx*, int batch, int* grid_out, int* items_per_cta_out, int* split_out);
+// The attention split around the recall: phase 1 covers the selected blocks that were already resident
+// (its result is the softmax state in `state`), phase 2 the blocks the step's recall list brings in, merged
+// with that state.  phase 0: everything in one call.
+struct pi_attn_phase {
+    int phase;
+    const pi_extent* rlist;
+    int rcap;
+    const int32_t* rcount;
+    float* state;
+};
+bool pi_attn_phased_fits(const pi_ctx*, int batch);
+long long pi_attn_state_floats(const pi_ctx*, int batch);
 int pi_launch_attn_headmajor(pi_ctx*, int batch, const void* q, const void* pool, const int32_t* sel_slots,
                              const int32_t* sel_blocks, const int32_t* sel_count, const int32_t* ctx_len,
-                             void* out, float* lse, int headwise, cudaStream_t);
+                             void* out, float* lse, int headwise, const pi_attn_phase* phase, cudaStream_t);
 int pi_launch_append(pi_ctx*, int h_star, int batch, uint32_t step, const void* k_new, const void* v_new,
                      const int32_t* ctx_len, void* host_kv, int64_t host_stride, void* pool, int32_t* table,
                      int32_t* slot_block, uint32_t* slot_stamp, void* digest, const int32_t* page_table,

@@ -105,6 +105,32 @@ class RecallPath:
         self.attention(layer, buf, q, ctx_len, out, lse)
 
 
+    def layer_step_split(self, layer: int, step: int, buf: LayerBuffers, q: torch.Tensor, ctx_len: torch.Tensor,
+                         host_kv: torch.Tensor, out: torch.Tensor, state: torch.Tensor, fused: bool = True) -> None:
+        """The layer's chain with the attention split around the recall: selection and diff on the current
+        stream, the resident blocks' share of the attention beside the recall on the side stream, the recalled
+        blocks' share on the current stream once the recall has landed."""
+        pi = self.pi
+        main = torch.cuda.current_stream()
+        if fused:
+            pi.score_select_diff(layer, step, q, buf.digest, ctx_len, buf.sel_blocks, buf.sel_count, buf.block_table,
+                                 buf.slot_block, buf.slot_stamp, buf.sel_slots, buf.recall_list, buf.recall_count,
+                                 scores=buf.scores)
+        else:
+            pi.score_select(layer, q, buf.digest, ctx_len, buf.sel_blocks, buf.sel_count, buf.scores)
+            pi.diff_misses(layer, step, ctx_len, buf.sel_blocks, buf.sel_count, buf.block_table, buf.slot_block,
+                           buf.slot_stamp, buf.sel_slots, buf.recall_list, buf.recall_count)
+        self._ev_in.record(main)
+        self.side.wait_event(self._ev_in)
+        pi.sparse_decode_attn_resident(layer, q, buf.pool, buf.sel_slots, buf.sel_blocks, buf.sel_count, ctx_len,
+                                       buf.recall_list, buf.recall_count, state, stream=self.side)
+        self._ev_recall.record(self.side)
+        pi.recall_gather_scatter(layer, host_kv, buf.pool, buf.recall_list, buf.recall_count)
+        main.wait_event(self._ev_recall)
+        pi.sparse_decode_attn_recalled(layer, q, buf.pool, buf.sel_slots, buf.sel_blocks, buf.sel_count, ctx_len,
+                                       buf.recall_list, buf.recall_count, state, out)
+
+
 class StageTimer:
     """CUDA events around each call of a decode step, on the stream the call runs on.
 
@@ -114,7 +140,7 @@ class StageTimer:
     afterwards (`light_summary`).  Extra events between the kernels of the recall streams cost
     the pipelined step about 6 % of its rate, which is why the timed region uses this form."""
 
-    STAGES = ("append", "select_diff", "score_select", "diff", "recall", "attn")
+    STAGES = ("append", "select_diff", "score_select", "diff", "recall", "attn_resident", "attn")
 
     def __init__(self, stages=None, light: bool = False):
         self.stages = tuple(stages) if stages else self.STAGES
@@ -216,8 +242,11 @@ class DecodeSession:
 
     def __init__(self, pi: PulseInfer, batch: int, n_layers: int, host_layers: Optional[int] = None,
                  device="cuda", keep_scores: bool = False, paged: bool = False, page_seed: int = 0,
-                 recall_streams: int = 2, fused_select_diff: bool = True):
+                 recall_streams: int = 2, fused_select_diff: bool = True, split_attention: bool = False):
         c = pi.cfg
+        # attention split around the recall: the resident blocks' share runs beside the recall (in the serial
+        # form on a stream of its own), the recalled blocks' share after it
+        self.split_attention = split_attention
         self.fused_select_diff = fused_select_diff     # selection + diff in one launch (pi_score_select_diff)
         self.pi, self.batch, self.n_layers = pi, batch, n_layers
         self.host_layers = n_layers if host_layers is None else max(1, min(host_layers, n_layers))
@@ -241,8 +270,10 @@ class DecodeSession:
         self._ev_diff = [torch.cuda.Event() for _ in range(n_layers)]
         self._ev_recall = [torch.cuda.Event() for _ in range(n_layers)]
         self._ev_attn = [torch.cuda.Event() for _ in range(n_layers)]
+        self._ev_res = [torch.cuda.Event() for _ in range(n_layers)]
         self._ev_start = torch.cuda.Event()
         self._path = RecallPath(pi)
+        self._attn_state = pi.attn_state(batch, self.device) if split_attention else None
         self.step_count = 0
         self._copy_s = None                  # copy stream and double buffers of the end-to-end form (made on first use)
         self._host_graph = None
@@ -354,18 +385,43 @@ class DecodeSession:
                 pi.diff_misses(l, step, self.ctx_len, b.sel_blocks, b.sel_count, b.block_table, b.slot_block,
                                b.slot_stamp, b.sel_slots, b.recall_list, b.recall_count, stream=sel_s)
                 t2 = tm.mark(sel_s) if tm and tm.wants("diff") else None
-            if overlapped:
+            split = self.split_attention
+            if split and self._attn_state is None:
+                self._attn_state = pi.attn_state(self.batch, self.device)
+            if overlapped or split:
                 evd.record(sel_s)
+            if overlapped:
                 rec_s.wait_event(evd)
+            # the resident blocks' share of a split attention runs beside the recall: on the attention stream in the
+            # pipelined form; in the serial form on the side stream, so that the chain select -> recall -> rest of
+            # the attention stays on one stream (dependent launches on a stream follow each other far more closely
+            # than launches that wait for another stream's event)
+            res_s = main if overlapped else self.side
+            if split:
+                res_s.wait_event(evd)
+                ta0 = tm.mark(res_s) if tm and tm.wants("attn_resident") else None
+                pi.sparse_decode_attn_resident(l, q[l], b.pool, b.sel_slots, b.sel_blocks, b.sel_count, self.ctx_len,
+                                               b.recall_list, b.recall_count, self._attn_state, stream=res_s)
+                if ta0 is not None:
+                    tm.add("attn_resident", ta0, tm.mark(res_s))
+                if not overlapped:
+                    evs = torch.cuda.Event() if capturing else self._ev_res[l]
+                    evs.record(res_s)
             t2r = tm.mark(rec_s) if tm and tm.wants("recall") else None
             pi.recall_gather_scatter(l, host, b.pool, b.recall_list, b.recall_count, page_table=pt, stream=rec_s)
             t3 = tm.mark(rec_s) if tm and tm.wants("recall") else None
             if overlapped:
                 evr.record(rec_s)
                 main.wait_event(evr)
+            elif split:
+                main.wait_event(evs)
             t4 = tm.mark(main) if tm and tm.wants("attn") else None
-            pi.sparse_decode_attn(l, q[l], b.pool, b.sel_slots, b.sel_blocks, b.sel_count, self.ctx_len,
-                                  out[l], None, stream=main)
+            if split:
+                pi.sparse_decode_attn_recalled(l, q[l], b.pool, b.sel_slots, b.sel_blocks, b.sel_count, self.ctx_len,
+                                               b.recall_list, b.recall_count, self._attn_state, out[l], stream=main)
+            else:
+                pi.sparse_decode_attn(l, q[l], b.pool, b.sel_slots, b.sel_blocks, b.sel_count, self.ctx_len,
+                                      out[l], None, stream=main)
             t5 = tm.mark(main) if tm and tm.wants("attn") else None
             if overlapped:
                 eva.record(main)

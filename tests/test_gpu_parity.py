@@ -534,6 +534,96 @@ def test_both_attention_forms_on_the_bench_shapes(mode):
     assert torch.equal(outs[0], outs[1])
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_attention_split_around_the_recall_random_shapes(seed):
+    """The resident blocks' share of the attention beside the recall, the recalled blocks' share after it:
+    the pair gives the oracle's attention on random shapes (KV heads, group sizes, block sizes, ragged and
+    empty sequences, first step with an almost empty pool = nearly everything recalled, later steps with few
+    misses), in the head-major form where it applies and through the fallback (the flat form) where not."""
+    from tests.parity import make_case, run_and_compare
+    rng = np.random.default_rng(7000 + seed)
+    Hkv = int(rng.choice([1, 2, 4, 8]))
+    G = int(rng.choice([1, 2, 4, 8, 16]))
+    B = int(rng.choice([16, 32, 64]))
+    batch = int(rng.integers(1, 6))
+    nb = int(rng.integers(12, 120))
+    sink = int(rng.choice([0, 16]))
+    local = int(rng.choice([0, 128]))
+    pinned = (-(-sink // B) if sink else 0) + (max(1, local // B) if local else 0)
+    K = int(rng.integers(pinned + 1, pinned + 40))
+    cfg = tiny_config(batch=batch, ctx=nb * B - int(rng.integers(0, B)), n_q_heads=Hkv * G, n_kv_heads=Hkv,
+                      block_tokens=B, budget_blocks=K, resident_frac=float(rng.choice([0.0, 0.3, 0.9])),
+                      sink_tokens=sink, local_tokens=local, seed=300 + seed)
+    lens = [int(rng.integers(0, cfg.ctx + 1)) for _ in range(batch)]
+    lens[0] = cfg.ctx
+    case = make_case(cfg, steps=3, ctx_len=np.asarray(lens), fill=float(rng.choice([0.0, 0.5, 1.0])))
+    mode = int(rng.choice([0, 1, 2]))                          # 1: the flat form, i.e. the fallback of the pair
+    ctas = int(rng.choice([0, 1, 3, 7])) if mode == 2 else 0
+    run_and_compare(case, steps=3, split=True, pi_kwargs=dict(attn_mode=mode, attn_ctas=ctas))
+
+
+@pytest.mark.parametrize("name,kw,pikw", [("c2", dict(n_layers=2), {}), ("c4", dict(n_layers=2), {}),
+                                          ("c3", dict(n_layers=1, batch=20), dict(attn_mode=2))])
+def test_attention_split_around_the_recall_on_the_bench_shapes(name, kw, pikw):
+    """The bench's shapes (c2: one CTA per item; c4: an item shared by a cluster of two CTAs; c3: block 32,
+    several items per CTA), pipelined session with the split attention against the oracle on sampled
+    sequences; the outputs also agree with the unsplit attention to a bf16 rounding step, and the split
+    repeats bit for bit."""
+    from tests.parity import run_session_sampled
+    cfg = get_config(name).replace(**kw)
+    seqs = [0, cfg.batch // 2, cfg.batch - 1]
+    outs = [run_session_sampled(cfg, steps=2, sample_seqs=seqs, return_out=True, split=sp, pi_kwargs=pikw)["out"].float()
+            for sp in (True, True, False)]
+    assert torch.equal(outs[0], outs[1])
+    gap = (outs[0] - outs[2]).abs()
+    assert float((gap / outs[2].abs().clamp_min(1.0)).max()) <= 2.0 ** -7, float(gap.max())
+
+
+def test_the_resident_share_reads_no_slot_that_the_recall_is_filling():
+    """Between the diff and the recall every destination slot of the recall list is overwritten with
+    large values; the first call of the split attention runs on that pool, then the recall, then the second
+    call.  Had the first call read one of those slots, the result would be far off the unsplit attention."""
+    from tests.parity import make_case
+    from paper_2609_34555_b200 import PulseInfer
+    from paper_2609_34555_b200.runner import LayerBuffers, RecallPath
+    cfg = tiny_config(batch=3, ctx=96 * 16 - 5, n_q_heads=32, n_kv_heads=8, budget_blocks=24, resident_frac=0.5, seed=11)
+    case = make_case(cfg, steps=3, ctx_len=np.asarray([cfg.ctx, 700, cfg.ctx - 40]))
+    dev = torch.device("cuda:0")
+    pi = PulseInfer.from_workload(cfg)
+    path = RecallPath(pi)
+    buf = LayerBuffers(pi, cfg.batch, dev)
+    ctx_d = torch.from_numpy(case.ctx_len).to(dev)
+    path.prepare_layer(0, buf, case.kv, ctx_d, torch.from_numpy(case.resident).to(dev))
+    state = pi.attn_state(cfg.batch, dev)
+    out = torch.zeros((cfg.batch, cfg.n_q_heads, cfg.head_dim), dtype=torch.bfloat16, device=dev)
+    plain = torch.zeros_like(out)
+    filled = 0
+    for t in range(3):
+        q = case.q[t].to(dev)
+        pi.score_select_diff(0, t + 1, q, buf.digest, ctx_d, buf.sel_blocks, buf.sel_count, buf.block_table, buf.slot_block,
+                             buf.slot_stamp, buf.sel_slots, buf.recall_list, buf.recall_count)
+        torch.cuda.synchronize()
+        lst, cnt = buf.recall_list.cpu().numpy(), buf.recall_count.cpu().numpy()
+        for s in range(cfg.batch):
+            for e in range(int(cnt[s])):
+                _, dst, n, _ = lst[s, e]
+                buf.pool[s, dst:dst + n] = 100.0
+                filled += int(n)
+        pi.sparse_decode_attn_resident(0, q, buf.pool, buf.sel_slots, buf.sel_blocks, buf.sel_count, ctx_d,
+                                       buf.recall_list, buf.recall_count, state)
+        torch.cuda.synchronize()
+        pi.recall_gather_scatter(0, case.kv, buf.pool, buf.recall_list, buf.recall_count)
+        pi.sparse_decode_attn_recalled(0, q, buf.pool, buf.sel_slots, buf.sel_blocks, buf.sel_count, ctx_d,
+                                       buf.recall_list, buf.recall_count, state, out)
+        pi.sparse_decode_attn(0, q, buf.pool, buf.sel_slots, buf.sel_blocks, buf.sel_count, ctx_d, plain)
+        torch.cuda.synchronize()
+        assert pi.status()[0] == 0
+        gap = (out.float() - plain.float()).abs() / plain.float().abs().clamp_min(1.0)
+        assert float(gap.max()) <= 2.0 ** -7, (t, float(gap.max()))
+    assert filled > 0
+    pi.close()
+
+
 def test_pipelined_session_with_append_on_two_layers():
     """DecodeSession's three-stream step with a token appended to every layer each step; the
     context crosses a block boundary on the way."""
