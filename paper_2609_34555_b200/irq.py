@@ -174,11 +174,16 @@ def simulate(mode: str, offload_layers: int = 64, t_io=400.0, **kw):
 # ------------------------------------------------------------------------------ CUDA back end
 class CudaOffload:
     """The offload batch on the GPU: DecodeSession buffers, selection + diff on stream A, recall
-    on stream B, attention (+ an FFN stand-in) on the compute stream."""
+    on stream B, attention (+ an FFN stand-in) on the compute stream.  split_attention: the resident
+    blocks' share of the attention is issued with the recall (stream A, behind the diff) and only the
+    recalled blocks' share is left for the moment the batch gets the GPU back."""
 
-    def __init__(self, sess, q_all, ffn):
+    def __init__(self, sess, q_all, ffn, split_attention: bool = False):
         import torch
         self.torch, self.sess, self.q_all, self.ffn = torch, sess, q_all, ffn
+        self.split = split_attention
+        self._state = sess.pi.attn_state(sess.batch, sess.device) if split_attention else None
+        self._resident_done = None
         self.compute_stream = torch.cuda.current_stream(sess.device)
         self.step = 0
         self._marks = []
@@ -202,6 +207,11 @@ class CudaOffload:
         pi.recall_gather_scatter(l, s.host_region(l), b.pool, b.recall_list, b.recall_count, stream=s.side2)
         io = self.torch.cuda.Event(enable_timing=True)
         io.record(s.side2)
+        if self.split:
+            pi.sparse_decode_attn_resident(l, q, b.pool, b.sel_slots, b.sel_blocks, b.sel_count, s.ctx_len,
+                                           b.recall_list, b.recall_count, self._state, stream=s.side)
+            self._resident_done = self.torch.cuda.Event()
+            self._resident_done.record(s.side)
         return io
 
     def compute(self, layer: int, io) -> None:
@@ -212,8 +222,13 @@ class CudaOffload:
         start = self.torch.cuda.Event(enable_timing=True)
         start.record(self.compute_stream)
         self._marks.append((io, start))
-        pi.sparse_decode_attn(l, q, b.pool, b.sel_slots, b.sel_blocks, b.sel_count, s.ctx_len, s.out[l], None,
-                              stream=self.compute_stream)
+        if self.split:
+            self.compute_stream.wait_event(self._resident_done)
+            pi.sparse_decode_attn_recalled(l, q, b.pool, b.sel_slots, b.sel_blocks, b.sel_count, s.ctx_len,
+                                           b.recall_list, b.recall_count, self._state, s.out[l], stream=self.compute_stream)
+        else:
+            pi.sparse_decode_attn(l, q, b.pool, b.sel_slots, b.sel_blocks, b.sel_count, s.ctx_len, s.out[l], None,
+                                  stream=self.compute_stream)
         self.ffn()
 
     def drain(self) -> None:
@@ -249,7 +264,7 @@ class CudaNormal:
 
 
 def run_on_gpu(offload_layers: int = 256, normal_batch: int = 64, normal_ctx: int = 4096, layers: int = 8,
-               recall_ctas: int = 0) -> list:
+               recall_ctas: int = 0, split_attention: bool = False) -> list:
     import numpy as np
     import torch
     sys.path.insert(0, str(Path(__file__).resolve().parent.parent))
@@ -289,7 +304,7 @@ def run_on_gpu(offload_layers: int = 256, normal_batch: int = 64, normal_ctx: in
     ffn_o = lambda: torch.matmul(torch.matmul(xo, w1), w2)
     out = []
     for mode in MODES:
-        off = CudaOffload(sess, q_all, ffn_o)
+        off = CudaOffload(sess, q_all, ffn_o, split_attention=split_attention)
         off.step = sess.step_count
         nor = CudaNormal(npi, nbuf, nq, nctx, nout, ffn_n, 32)
         rep = IrqScheduler(off, nor, mode).run(offload_layers)
@@ -305,6 +320,9 @@ if __name__ == "__main__":
     ap.add_argument("--normal-batch", type=int, default=64)
     ap.add_argument("--normal-ctx", type=int, default=4096)
     ap.add_argument("--recall-ctas", type=int, default=10, help="one recall launch at a time here: 10 CTAs (the library default of 5 is sized for two launches side by side)")
+    ap.add_argument("--split-attention", action="store_true",
+                    help="the resident blocks' share of the offload batch's attention is issued with the recall")
     a = ap.parse_args()
-    for r in run_on_gpu(a.offload_layers, a.normal_batch, a.normal_ctx, recall_ctas=a.recall_ctas):
+    for r in run_on_gpu(a.offload_layers, a.normal_batch, a.normal_ctx, recall_ctas=a.recall_ctas,
+                        split_attention=a.split_attention):
         print(json.dumps(r))
