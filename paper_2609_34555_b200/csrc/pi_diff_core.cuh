@@ -49,6 +49,11 @@ struct Smem {
     const int32_t* table_s;
     int* warp_tot;                  // [2][NT / 32]
     int* n_cand;
+    // Optional (cluster form): all C slots in eviction order, (stamp, slot) ascending, written into this CTA's
+    // shared memory by another CTA of the cluster, which arrives on the mbarrier `lru_bar` when it is done.
+    const unsigned short* lru_order;
+    uint32_t lru_bar;               // shared-memory address of that mbarrier (phase 0)
+    long long lru_wait;             // bound of the wait in cycles
 };
 
 // Bytes of the arrays above (without the key union), and of the union.
@@ -76,6 +81,7 @@ __device__ __forceinline__ Smem carve(unsigned char* base, int K, int C) {
     m.stp = reinterpret_cast<uint32_t*>(m.sb + C);
     m.used = reinterpret_cast<unsigned char*>(m.stp + C);
     m.keys = nullptr; m.table_s = nullptr; m.warp_tot = nullptr; m.n_cand = nullptr;
+    m.lru_order = nullptr; m.lru_bar = 0; m.lru_wait = 0;
     return m;
 }
 
@@ -122,12 +128,63 @@ __device__ __forceinline__ void diff_sequence(const SeqArgs& a, const Smem& m, p
     }
     __syncthreads();
 
+    // 2'. The slots in eviction order came from another CTA of the cluster: the victims are the first n_miss of
+    //     them that may be evicted (not holding a block of this selection, not holding a sink or local block).
+    bool use_order = m.lru_order != nullptr && n_miss > 0 && n_miss <= RANK_MAX_MISSES;
+    bool too_small = false;
+    int n_cand = 0;
+    if (use_order) {
+        bool ok = false;
+        {
+            uint32_t done = 0;
+            const long long t0 = clock64();
+            for (;;) {
+                asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                             : "=r"(done) : "r"(m.lru_bar), "r"(0u) : "memory");
+                if (done || clock64() - t0 > m.lru_wait) break;
+            }
+            ok = done != 0;
+        }
+        use_order = __syncthreads_and(ok) != 0;             // (a wait that ran out: the victims are found the other way)
+    }
+    if (use_order) {
+        int found = 0;
+        for (int base = 0, it = 0; base < a.C && found < n_miss; base += NT, ++it) {
+            const int r = base + tid;
+            bool cand = false;
+            int s = 0;
+            if (r < a.C) {
+                s = m.lru_order[r];
+                const int b = m.sb[s];
+                const bool pinned = b >= 0 && (b < a.n_sink || b >= a.n_blocks - a.n_local);
+                cand = b < 0 || (!m.used[s] && !pinned);
+            }
+            const unsigned bal = __ballot_sync(0xffffffffu, cand);
+            int* wt = m.warp_tot + (it & 1) * NW;
+            if (lane == 0) wt[warp] = __popc(bal);
+            __syncthreads();
+            int off = 0, tot = 0;
+#pragma unroll
+            for (int i = 0; i < NW; ++i) {
+                const int t = wt[i];
+                if (i < warp) off += t;
+                tot += t;
+            }
+            const int pos = found + off + __popc(bal & ((1u << lane) - 1u));
+            if (cand && pos < n_miss) m.vict[pos] = s;
+            found += tot;
+        }
+        n_cand = found;                                     // all candidates when there are too few of them
+        too_small = found < n_miss;
+        __syncthreads();
+    }
+
     // 2. victim candidates.  Ranking path: key = inverted stamp (older = larger), 0 for a slot that may not
     //    be evicted.  Sort path: (stamp, slot) in 64 bits, everything else sorts to the end.
     const bool rank_path = n_miss <= RANK_MAX_MISSES;
     unsigned long long* keys64 = reinterpret_cast<unsigned long long*>(m.keys);
     uint32_t kmin = 0xffffffffu, kmax = 0u;             // extremes of the candidates' ranking keys, found on the way
-    if (n_miss > 0) {
+    if (n_miss > 0 && !use_order) {
         int my_cand = 0;
 #pragma unroll 1
         for (int s = tid; s < (rank_path ? a.C : a.Cpad); s += NT) {
@@ -156,16 +213,20 @@ __device__ __forceinline__ void diff_sequence(const SeqArgs& a, const Smem& m, p
             sc.red_lo[warp] = kmin; sc.red_hi[warp] = kmax;
         }
     }
-    __syncthreads();
-    const int n_cand = *m.n_cand;
-    const bool too_small = n_cand < n_miss;
-    if (n_miss > 0) {
+    if (!use_order) {
+        __syncthreads();
+        n_cand = *m.n_cand;
+        too_small = n_cand < n_miss;
+    }
+    if (n_miss > 0 && !use_order) {
         kmin = __reduce_min_sync(0xffffffffu, lane < NW ? sc.red_lo[lane] : 0xffffffffu);
         kmax = __reduce_max_sync(0xffffffffu, lane < NW ? sc.red_hi[lane] : 0u);
     }
 
     if (n_miss > 0 && !too_small) {
-        if (rank_path) {
+        if (use_order) {
+            // (the victims are in m.vict already)
+        } else if (rank_path) {
             // 3a. the n_miss oldest candidates (ties to the lower slot), gathered in slot order, then
             //     ranked by (stamp ascending, slot ascending) against each other
             // (stamps repeat a lot: lanes that hit the same histogram bin add once; the slots that may not be

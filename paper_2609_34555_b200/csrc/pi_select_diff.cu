@@ -55,6 +55,10 @@ struct SDParams {
     uint32_t step;
     int C, Cpad, table_in_smem;
     unsigned key_bytes;            // bytes of the key region at the start of the dynamic shared memory
+    // eviction order prepared by the cluster's second CTA while the first one selects (fused form, clusters of 2+)
+    int lru_help;
+    unsigned order_off;            // byte offset of the order array (uint16 [C]) in the first CTA's dynamic shared memory
+    long long wait_cycles;
 };
 
 __device__ __forceinline__ unsigned cluster_ctarank() {
@@ -79,6 +83,9 @@ __device__ __forceinline__ uint32_t map_shared_rank(const void* p, unsigned rank
 __device__ __forceinline__ void st_shared_cluster(uint32_t addr, uint32_t v) {
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
+__device__ __forceinline__ void st_shared_cluster_u16(uint32_t addr, unsigned short v) {
+    asm volatile("st.shared::cluster.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
+}
 __device__ __forceinline__ void cp_async4(void* smem, const void* gmem) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem))), "l"(gmem) : "memory");
 }
@@ -95,6 +102,7 @@ score_select_cluster_kernel(SDParams p) {
     __shared__ int warp_tot[2 * SD_WARPS];
     __shared__ int s_ncand;
     __shared__ uint32_t s_mm[2 * SD_MAX_CLUSTER * SD_WARPS];       // first CTA: every scoring warp's smallest and largest middle key
+    __shared__ __align__(8) unsigned long long s_lru_bar;          // first CTA: the second CTA arrives here when the eviction order is written
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned rank = cluster_ctarank(), CL = cluster_nctarank();
@@ -184,9 +192,18 @@ score_select_cluster_kernel(SDParams p) {
                 }
             }
             if (tid == 0) s_ncand = 0;
+            if (tid == 0 && p.lru_help) {
+                asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(&s_lru_bar))), "r"(CL - 1u));
+                asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            }
         }
+    } else if (FUSED && p.lru_help) {
+        // the stamps of all slots, for the eviction order the other CTAs work out after their share of the scoring
+        // (their own dynamic shared memory is free: the keys go to the first CTA)
+        uint32_t* st = reinterpret_cast<uint32_t*>(smem_raw + static_cast<size_t>((p.C + 1) & ~1) * 8);
+        const uint32_t* stp = p.slot_stamp + static_cast<size_t>(seq) * p.C;
+        for (int s = tid; s < p.C; s += SD_THREADS) cp_async4(st + s, stp + s);
     }
-
     {
         pi_score::load_q_weights(p.q + (static_cast<size_t>(seq) * p.Hq + static_cast<size_t>(p.h_star) * p.G) * PI_HEAD_DIM,
                                  p.G, lane, w);
@@ -222,10 +239,48 @@ score_select_cluster_kernel(SDParams p) {
         st_shared_cluster(mm_remote, kmin);
         st_shared_cluster(mm_remote + 4u, kmax);
     }
-    if (FUSED && rank == 0) cp_async_wait_all();
+    if (FUSED && (rank == 0 || p.lru_help)) cp_async_wait_all();
     // all keys of the sequence are in the first CTA's shared memory once every CTA has arrived
     cluster_arrive_release();
     cluster_wait_acquire();
+    if (FUSED && rank != 0 && p.lru_help) {
+        // ---------------- eviction order for the first CTA's diff, worked out while that CTA selects: position of
+        // slot s = number of slots before it in (stamp, slot) order, by counting.  The CL - 1 other CTAs take every
+        // (CL - 1)-th slot each; four lanes share the comparisons of one slot.  The positions go straight into the
+        // first CTA's shared memory, then every CTA arrives once on its mbarrier.
+        __syncthreads();                                   // every thread's share of the stamps has landed
+        const int Cq = (p.C + 1) & ~1;
+        unsigned long long* k64 = reinterpret_cast<unsigned long long*>(smem_raw);
+        const uint32_t* st = reinterpret_cast<const uint32_t*>(smem_raw + static_cast<size_t>(Cq) * 8);
+        for (int u = tid; u < Cq; u += SD_THREADS)
+            k64[u] = u < p.C ? ((static_cast<unsigned long long>(st[u]) << 32) | static_cast<unsigned>(u)) : ~0ull;
+        __syncthreads();
+        const uint32_t order_remote = map_shared_rank(smem_raw + p.order_off, 0);
+        const int parts = static_cast<int>(CL) - 1, part = static_cast<int>(rank) - 1;
+        const int n_mine = (p.C - part + parts - 1) / parts;                  // slots part, part + parts, ...
+        const int qd = tid & 3, pairs = Cq >> 1;
+        for (int i0 = 0; i0 < n_mine; i0 += SD_THREADS / 4) {
+            const int i = i0 + (tid >> 2);
+            const int s = part + i * parts;
+            const unsigned long long mine = i < n_mine ? k64[s] : 0ull;
+            int before = 0;
+#pragma unroll 4
+            for (int u2 = qd; u2 < pairs; u2 += 4) {
+                const ulonglong2 v = reinterpret_cast<const ulonglong2*>(k64)[u2];
+                before += (v.x < mine ? 1 : 0) + (v.y < mine ? 1 : 0);
+            }
+            before += __shfl_xor_sync(0xffffffffu, before, 1);
+            before += __shfl_xor_sync(0xffffffffu, before, 2);
+            if (qd == 0 && i < n_mine)
+                st_shared_cluster_u16(order_remote + 2u * static_cast<uint32_t>(before), static_cast<unsigned short>(s));
+        }
+        __syncthreads();
+        if (tid == 0) {
+            const uint32_t bar_remote = map_shared_rank(&s_lru_bar, 0);
+            asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_remote) : "memory");
+        }
+        return;
+    }
     if (rank != 0) return;
 
     // ---------------- selection: sink and local blocks always, the k_mid best middle blocks, ties to the lower index
@@ -269,8 +324,23 @@ score_select_cluster_kernel(SDParams p) {
     m.table_s = p.table_in_smem ? s_table : nullptr;
     m.warp_tot = warp_tot;
     m.n_cand = &s_ncand;
+    if (p.lru_help && CL >= 2) {
+        m.lru_order = reinterpret_cast<const unsigned short*>(smem_raw + p.order_off);
+        m.lru_bar = static_cast<uint32_t>(__cvta_generic_to_shared(&s_lru_bar));
+        m.lru_wait = p.wait_cycles;
+    }
     __syncthreads();
     pi_diff::diff_sequence<SD_THREADS>(a, m, sc);
+    if (p.lru_help && CL >= 2 && tid == 0) {
+        // The second CTA writes the eviction order into this CTA's shared memory whether or not the diff needed it
+        // (no misses, or too many for the ranked path): this CTA stays until that CTA has arrived.
+        const long long t0 = clock64();
+        uint32_t done = 0;
+        while (!done && clock64() - t0 <= p.wait_cycles)
+            asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                         : "=r"(done) : "r"(m.lru_bar), "r"(0u) : "memory");
+        if (!done) pi_report(p.st, PI_ERR_TIMEOUT, PI_STAGE_DIFF, seq, 0, 0);
+    }
 }
 
 // Clusters of `cluster` CTAs of this kernel that the device holds at once (0 if the query fails).
@@ -328,6 +398,13 @@ int pi_launch_select_cluster(pi_ctx* c, int h_star, int batch, const void* q, co
         if (smem + row <= SD_SMEM_LIMIT) { p.table_in_smem = 1; smem += row; }
     }
     p.key_bytes = static_cast<unsigned>(key_bytes);
+    // room for the eviction order (uint16 per slot) the second CTA of a cluster hands to the first
+    p.lru_help = 0; p.order_off = 0; p.wait_cycles = c->wait_limit_cycles;
+    const bool order_room = fused && p.C <= 1024 && smem + 2 * static_cast<size_t>(p.C) + 16 <= SD_SMEM_LIMIT;
+    if (order_room) {
+        p.order_off = static_cast<unsigned>((smem + 15) & ~size_t(15));
+        smem = p.order_off + 2 * static_cast<size_t>(p.C);
+    }
     auto kern = fused ? score_select_cluster_kernel<true> : score_select_cluster_kernel<false>;
     if (smem > 36 * 1024)
         PI_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
@@ -344,6 +421,7 @@ int pi_launch_select_cluster(pi_ctx* c, int h_star, int batch, const void* q, co
         if (batch <= resident[log2c]) { cluster = cl; break; }
     }
     p.cpc = (n_chunks + cluster - 1) / cluster;
+    p.lru_help = (order_room && cluster >= 2) ? 1 : 0;
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(batch * cluster);
     lc.blockDim = dim3(SD_THREADS);
