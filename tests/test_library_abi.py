@@ -60,3 +60,6 @@ def test_null_arguments_are_rejected():
     assert lib.pi_destroy(None) == -1
     assert lib.pi_score_select(None, 0, 1, None, None, None, None, None, None, None) == -1
     assert lib.pi_get_status(None, None) == -1
+    assert lib.pi_sparse_decode_attn_resident(None, 0, 1, None, None, None, None, None, None, None, 1, None, None, None) == -1
+    assert lib.pi_sparse_decode_attn_recalled(None, 0, 1, None, None, None, None, None, None, None, 1, None, None, None, None) == -1
+    assert lib.pi_attn_state_bytes(None, 1) == -1
