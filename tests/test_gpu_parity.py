@@ -443,6 +443,19 @@ def test_largest_supported_block_count_and_wide_budget():
     assert stats["misses"][0] > 100
 
 
+def test_more_than_512_misses_in_the_fused_launch_take_the_sorting_path():
+    """A 640-block budget against a pool of 1 024 slots that holds almost none of the selection: about 600
+    misses per step, beyond what the ranked victim search covers.  In the one-launch form the cluster's other
+    CTAs still prepare the eviction order (the pool is small enough for it); the first CTA ignores it, sorts,
+    and must not leave before they are done."""
+    from tests.parity import make_case, run_and_compare
+    cfg = tiny_config(batch=2, ctx=131072, n_q_heads=8, n_kv_heads=2, budget_blocks=640, resident_frac=1024 / 8192)
+    assert cfg.n_blocks == 8192 and cfg.pool_slots == 1024
+    case = make_case(cfg, steps=2)
+    stats = run_and_compare(case, steps=2)
+    assert max(stats["misses"]) > 512
+
+
 def test_averaged_and_headwise_selection_strategies():
     from tests.parity import run_strategies_and_compare
     cfg = tiny_config(batch=2, ctx=3000, n_q_heads=16, n_kv_heads=4, budget_blocks=32, resident_frac=0.3)
