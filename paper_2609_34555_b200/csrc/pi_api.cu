@@ -50,7 +50,7 @@ extern "C" int pi_create(const pi_config* cfg, pi_ctx** out) {
     std::memset(c, 0, sizeof(*c));
     c->cfg = *cfg;
     for (int i = 0; i < 2; ++i)
-        for (int j = 0; j < 4; ++j) c->sd_resident_clusters[i][j] = -1;
+        for (int j = 0; j < 5; ++j) c->sd_resident_clusters[i][j] = -1;
     c->solo_head = static_cast<int32_t*>(std::malloc(sizeof(int32_t) * cfg->n_layers));
     std::memcpy(c->solo_head, cfg->solo_head, sizeof(int32_t) * cfg->n_layers);
     c->cfg.solo_head = c->solo_head;

@@ -85,7 +85,7 @@ struct pi_ctx {
     int pool_map_headwise;       // box of the cached map: all KV heads of a block (0) or one head (1)
     void* encode_tiled_fn;
     // clusters of 2^i CTAs of the selection kernel that are resident at once, [plain | fused][i]; -1 = not asked yet
-    int sd_resident_clusters[2][4];
+    int sd_resident_clusters[2][5];
 };
 
 struct pi_status_ref {

@@ -30,7 +30,7 @@ constexpr int SD_THREADS = SD_THREADS_OVERRIDE;
 constexpr bool SD_TWO_SETS = SD_THREADS <= 256;            // two register sets of loads per lane (else one)
 constexpr int SD_WARPS = SD_THREADS / 32;
 constexpr int SD_CHUNK = SD_WARPS * BLOCKS_PER_WARP;      // 64 blocks (32 KB of digests); a CTA loads two chunks a round
-constexpr int SD_MAX_CLUSTER = 8;
+constexpr int SD_MAX_CLUSTER = 16;                        // 16 is beyond the portable cluster size: taken only where the device holds enough of them
 constexpr size_t SD_SMEM_LIMIT = 200 * 1024;              // dynamic shared memory the kernel may ask for
 
 struct SDParams {
@@ -408,16 +408,25 @@ int pi_launch_select_cluster(pi_ctx* c, int h_star, int batch, const void* q, co
     auto kern = fused ? score_select_cluster_kernel<true> : score_select_cluster_kernel<false>;
     if (smem > 36 * 1024)
         PI_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    // Cluster size: the largest power of two <= 8 that leaves no CTA without blocks and lets the clusters of all
+    // Cluster size: the largest power of two <= 16 that leaves no CTA without blocks and lets the clusters of all
     // sequences be resident at once (a cluster that has to wait for another one to finish doubles the
     // latency of the call); what the device holds is asked once per shape and kept.
     const int n_chunks = (cfg.max_blocks + SD_CHUNK - 1) / SD_CHUNK;
     int* resident = c->sd_resident_clusters[fused ? 1 : 0];
     int cluster = 1;
-    for (int log2c = 3; log2c >= 1; --log2c) {
+    for (int log2c = 4; log2c >= 1; --log2c) {
         const int cl = 1 << log2c;
         if (cl > n_chunks) continue;                               // more CTAs than chunks
-        if (resident[log2c] < 0) resident[log2c] = resident_clusters(kern, cl, smem);
+        // a cluster of 16 only for long sequences: below four chunks per CTA the extra CTAs of a sequence gain nothing
+        if (cl == 16 && n_chunks < 64) continue;
+        if (resident[log2c] < 0) {
+            if (cl == 16 && cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+                (void)cudaGetLastError();
+                resident[log2c] = 0;
+            } else {
+                resident[log2c] = resident_clusters(kern, cl, smem);
+            }
+        }
         if (batch <= resident[log2c]) { cluster = cl; break; }
     }
     p.cpc = (n_chunks + cluster - 1) / cluster;
