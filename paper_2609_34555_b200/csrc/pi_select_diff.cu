@@ -10,6 +10,11 @@
 // which is still in its shared memory, against the block table.  What the diff needs besides the
 // selection (the sequence's slot arrays and its table row) is fetched with asynchronous copies
 // while the scoring loads are in flight, so that no global round trip is left between the steps.
+// The cluster's other CTAs, idle once their keys are delivered, meanwhile work out the order in
+// which the pool's slots would be evicted (least recently selected first) and hand it to the first
+// CTA through its shared memory and an mbarrier: the victims of the diff are then the first
+// evictable slots of that order instead of a second top-k by the one CTA that is already the
+// launch's critical path.
 #include "pi_common.cuh"
 #include "pi_block_select.cuh"
 #include "pi_diff_core.cuh"
@@ -30,6 +35,11 @@ constexpr int SD_THREADS = SD_THREADS_OVERRIDE;
 constexpr bool SD_TWO_SETS = SD_THREADS <= 256;            // two register sets of loads per lane (else one)
 constexpr int SD_WARPS = SD_THREADS / 32;
 constexpr int SD_CHUNK = SD_WARPS * BLOCKS_PER_WARP;      // 64 blocks (32 KB of digests); a CTA loads two chunks a round
+// chunks a sequence must have before it gets a cluster of 16 CTAs (below four chunks per CTA the extra CTAs
+// gain nothing: measured at 32 chunks)
+#ifndef SD_CL16_MIN_CHUNKS
+#define SD_CL16_MIN_CHUNKS 64
+#endif
 constexpr int SD_MAX_CLUSTER = 16;                        // 16 is beyond the portable cluster size: taken only where the device holds enough of them
 constexpr size_t SD_SMEM_LIMIT = 200 * 1024;              // dynamic shared memory the kernel may ask for
 
@@ -418,7 +428,7 @@ int pi_launch_select_cluster(pi_ctx* c, int h_star, int batch, const void* q, co
         const int cl = 1 << log2c;
         if (cl > n_chunks) continue;                               // more CTAs than chunks
         // a cluster of 16 only for long sequences: below four chunks per CTA the extra CTAs of a sequence gain nothing
-        if (cl == 16 && n_chunks < 64) continue;
+        if (cl == 16 && n_chunks < SD_CL16_MIN_CHUNKS) continue;
         if (resident[log2c] < 0) {
             if (cl == 16 && cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
                 (void)cudaGetLastError();
