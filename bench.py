@@ -44,7 +44,7 @@ METRIC = "decode layer-steps/s (select+recall+attn); recall GB/s vs measured H2D
 # profiles/ (attn_kernel_c2.txt, score_select_kernel_c2.txt): same per-layer shapes as the bench
 # (recall_kernel: its reads cross the host link and its 5 MB of writes stay in L2 during the launch,
 # so DRAM sees next to nothing)
-NCU_DRAM_TRAFFIC = {"c2": {"recall_kernel": 21.0e3}}
+NCU_DRAM_TRAFFIC = {"c2": {"recall_kernel": 24.7e3}}
 FALLBACK_HBM_GBS = 6650.0
 
 
