@@ -41,10 +41,11 @@ import torch
 
 METRIC = "decode layer-steps/s (select+recall+attn); recall GB/s vs measured H2D peak"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
-# profiles/ (attn_kernel_c2.txt, score_select_kernel_c2.txt): same per-layer shapes as the bench
-# (recall_kernel: its reads cross the host link and its 5 MB of writes stay in L2 during the launch,
-# so DRAM sees next to nothing)
-NCU_DRAM_TRAFFIC = {"c2": {"recall_kernel": 24.7e3}}
+# profiles/ (attn_headmajor_kernel_c2.txt, score_select_cluster_kernel_c2.txt, recall_kernel_c2.txt): same
+# per-layer shapes as the bench (recall_kernel: its reads cross the host link and its 5 MB of writes stay
+# in L2 during the launch, so DRAM sees next to nothing; the attention's 4 MB of DRAM writes are write-backs
+# of lines that were dirty in L2 when the capture started, the kernel itself writes 131 KB)
+NCU_DRAM_TRAFFIC = {"c2": {"recall_kernel": 24.7e3, "attn_kernel": 134.42e6 + 4.2e6, "score_select_diff_kernel": 17.07e6}}
 FALLBACK_HBM_GBS = 6650.0
 
 
