@@ -203,6 +203,8 @@ int pi_diff_misses_devstep(pi_ctx* ctx, int layer, int batch, const uint32_t* st
  *                            An extent whose units reach beyond the sequence's pool region (C blocks) or,
  *                            in the block-major store, its host region (NB blocks) sets PI_ERR_INDEX_RANGE
  *                            in the status word (stage 3: list, extent, unit); those units are skipped.
+ *                            A list whose units add up to more than the pool region holds is skipped as a
+ *                            whole with PI_ERR_CAPACITY (stage 3: list, units, capacity).
  *   unit_stride_bytes        distance between consecutive units (0 = unit_bytes: units are contiguous)
  *   list_offset_bytes        list i starts (i % lists_per_seq) * list_offset_bytes into its sequence's
  *                            region, in the host store and in the pool alike (0 for the shared selection) */

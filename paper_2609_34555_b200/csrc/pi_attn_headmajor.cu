@@ -115,9 +115,13 @@ attn_headmajor_kernel(const __grid_constant__ CUtensorMap pool_map, AttnParams p
             if (n < 0 || n > p.rcap) n = 0;                 // (the recall kernel reports such a count)
             for (int e = tid; e < n; e += blockDim.x) {
                 const pi_extent x = p.rlist[static_cast<size_t>(seq) * p.rcap + e];
-                for (int u = 0; u < x.n_units; ++u) {
+                // (an extent that leaves the pool is the recall kernel's to report; here it is clipped, which also
+                // bounds the loop whatever the list holds)
+                if (x.dst_unit < 0 || x.dst_unit >= p.C) continue;
+                const int nu = min(x.n_units, p.C - x.dst_unit);
+                for (int u = 0; u < nu; ++u) {
                     const int slot = x.dst_unit + u;
-                    if (slot >= 0 && slot < p.C) atomicOr(&s_fresh[k * words + (slot >> 5)], 1u << (slot & 31));
+                    atomicOr(&s_fresh[k * words + (slot >> 5)], 1u << (slot & 31));
                 }
             }
         }

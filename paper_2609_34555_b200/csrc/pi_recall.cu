@@ -125,6 +125,12 @@ recall_kernel(RecallParams p) {
                 const pi_extent e = cached ? s_ext[s_eoff[l + 1] - 1] : p.list[static_cast<size_t>(l) * p.cap + n - 1];
                 u = static_cast<long long>(e.units_before) + e.n_units;
                 if (u < 0) u = 0;
+                // a list cannot move more units than its sequence's pool region holds: a larger total is a
+                // damaged list, and walking it would keep the kernel busy for nothing
+                if (u > p.pool_units) {
+                    if (blockIdx.x == 0) pi_report(p.st, PI_ERR_CAPACITY, PI_STAGE_RECALL, l, static_cast<int>(min(u, 0x7fffffffLL)), static_cast<int>(min(p.pool_units, 0x7fffffffLL)));
+                    u = 0;
+                }
             }
         }
         const long long off = block_scan_add(u, warp_tot, run);

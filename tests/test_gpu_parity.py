@@ -238,6 +238,21 @@ def test_recall_skips_and_reports_an_extent_that_leaves_the_pool_or_the_host_reg
                 want[1, dst + k] = kv[1, src + k]
         assert torch.equal(got.view(torch.int16), want.view(torch.int16))
         pi.clear_status()
+    # a damaged list (a billion units): skipped as a whole and reported, the other list is copied, the call returns at once
+    pool.zero_()
+    lst = torch.zeros((cfg.batch, cfg.budget_blocks, 4), dtype=torch.int32, device=dev)
+    lst[0, 0] = torch.tensor([3, 2, 2, 0])
+    lst[1, 0] = torch.tensor([1, 0, 1 << 30, 0])
+    cnt = torch.tensor([1, 1], dtype=torch.int32, device=dev)
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record(); pi.recall_gather_scatter(0, kv, pool, lst, cnt); t1.record()
+    torch.cuda.synchronize()
+    st = pi.status()
+    assert st[0] == -9 and st[1] == 3 and st[2] == 1 and st[4] == C, st
+    assert t0.elapsed_time(t1) < 50.0
+    want = torch.zeros_like(pool.cpu()); want[0, 2:4] = kv[0, 3:5]
+    assert torch.equal(pool.cpu().view(torch.int16), want.view(torch.int16))
+    assert bool((arena[~covered] == 0x5A).all()), "written outside the pool"
     pi.close()
 
 
