@@ -860,7 +860,8 @@ def test_layer_step_can_be_captured_into_a_cuda_graph_and_replayed():
     pi.close()
 
 
-def test_graph_replayed_decode_steps_match_eager_steps():
+@pytest.mark.parametrize("split", [False, True], ids=["attention in one call", "attention split around the recall"])
+def test_graph_replayed_decode_steps_match_eager_steps(split):
     """A whole pipelined decode step (three layers, all streams) captured once and replayed, with an
     eager step mixed in: outputs, tables and stamps equal those of a session stepped eagerly."""
     import torch
@@ -872,7 +873,7 @@ def test_graph_replayed_decode_steps_match_eager_steps():
     results = []
     for form in ("eager", "graph"):
         pi = PulseInfer.from_workload(cfg)
-        sess = DecodeSession(pi, cfg.batch, cfg.n_layers)
+        sess = DecodeSession(pi, cfg.batch, cfg.n_layers, split_attention=split)
         sess.ctx_len.fill_(cfg.ctx)
         for l in range(cfg.n_layers):
             kv = gen.make_kv(cfg, l, device=sess.device)
