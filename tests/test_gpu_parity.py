@@ -143,6 +143,17 @@ def test_full_size_config3_shapes_block_32_sampled():
     assert stats["misses"] > 0
 
 
+@pytest.mark.parametrize("B", [16, 64])
+def test_full_size_config5_shapes_batch_32_sampled(B):
+    """The recall-fragmentation config's layer (batch 32, 32 768 tokens; blocks of 16 tokens with a budget of
+    128 blocks, and blocks of 64 tokens with a budget of 32) in the bench's launch configuration: 256 work
+    items for the attention (two per CTA), 32 selection clusters; the oracle follows three sequences."""
+    from tests.parity import run_session_sampled
+    cfg = get_config("c5").replace(block_tokens=B, budget_blocks=max(128 * 16 // B, 16))
+    stats = run_session_sampled(cfg, steps=3, sample_seqs=[0, 17, 31])
+    assert stats["misses"] > 0
+
+
 def gen_pinned(cfg):
     from workloads import generate as gen
     return gen.pinned_blocks(cfg).tolist()
